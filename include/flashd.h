@@ -1,0 +1,167 @@
+/*
+ * flashd.h - C ABI of the FLASH-D attention forward library for NVIDIA B200
+ * (sm_100a).
+ *
+ * The library computes  O = softmax(scale * Q K^T) V  in the form of the
+ * paper "FLASH-D: FlashAttention with Hidden Softmax Division": the running
+ * output is a convex blend  o_i = o_{i-1} (1 - w_i) + v_i w_i  (Eq. out-final)
+ * whose weight  w_i = sigma(s_i - s_{i-1} + ln w_{i-1})  (Eq. w-last) absorbs
+ * the softmax division, so the output is normalised after every step, no
+ * running maximum is carried and no final division is made (Algorithm 3).
+ *
+ * Conventions shared by every entry point
+ *   - Tensors are contiguous [B, H, N, d] arrays, d innermost; q and o have
+ *     N = Nq, k and v have N = Nk.  The paper treats one head (Sec. II); B*H
+ *     independent heads are processed here.
+ *   - Unless an argument is documented as a HOST pointer, tensor pointers are
+ *     DEVICE pointers owned by the caller, 16-byte aligned.  The library keeps
+ *     no reference to them after the work queued on `stream` has finished.
+ *   - s = scale * dot(q, k).  The paper's score has no scale factor (Sec. II-A);
+ *     pass scale = 1 for the paper's definition, 1/sqrt(d) for transformers.
+ *   - causal != 0: key j is visible to query i iff j <= i (0-based indices).
+ *     Keys that a query cannot see are removed from its key sequence.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls enqueue work and return without synchronising, except where
+ *     stated.
+ *   - Every function returns a flashd_status (0 = success).  Arguments are
+ *     validated on the host before anything is launched; nothing is launched
+ *     when validation fails.  The library never aborts and never throws.
+ *   - There is no CPU fallback: without a CUDA device the calls return
+ *     FLASHD_ERR_CUDA.
+ */
+#ifndef FLASHD_H
+#define FLASHD_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FLASHD_OK = 0,
+    FLASHD_ERR_NULL = 1,        /* a required pointer is NULL                          */
+    FLASHD_ERR_SHAPE = 2,       /* a size is <= 0, or scale is not finite              */
+    FLASHD_ERR_UNSUPPORTED = 3, /* head size / dtype / mode not built                  */
+    FLASHD_ERR_ALIGN = 4,       /* a tensor pointer is not 16-byte aligned             */
+    FLASHD_ERR_WORKSPACE = 5,   /* workspace too small or split count out of range     */
+    FLASHD_ERR_CUDA = 6,        /* a CUDA runtime / driver call failed                 */
+    FLASHD_ERR_TIMEOUT = 7      /* a bounded wait inside a kernel ran out              */
+} flashd_status;
+
+typedef enum { FLASHD_BF16 = 0, FLASHD_F32 = 1 } flashd_dtype;
+
+/* Upper bound on num_splits accepted by the split-K entry points. */
+#define FLASHD_MAX_SPLITS 64
+
+/* ------------------------------------------------------------------------
+ * Tiled tensor-core forward (bf16 in, fp32 accumulate, bf16 out).
+ *
+ * Computes Algorithm 3 with keys grouped in tiles of 128: for each tile the
+ * weights of its keys and the weight (1 - W) of the old output follow from
+ * Eq. (w-last) applied to the tile as one "super-key" whose score is the
+ * log-sum-exp L_T of the tile's scores:
+ *     L_new = L_T - ln sigma(L_T - L_old),  P_j = exp(s_j - L_new),
+ *     alpha = exp(L_old - L_new),           O <- alpha O + P V_tile,
+ * which is Eq. (out-final) for the group.  The carried state per query row is
+ * L alone (= s_i - ln w_i of the paper).  S = Q K^T and P V run on the 5th
+ * generation tensor cores (tcgen05.mma, accumulators in tensor memory).
+ *
+ * q, o: [B,H,Nq,d] bf16; k, v: [B,H,Nk,d] bf16.  d must be 64 or 128.
+ * o must not overlap q, k or v.  Returns after the launch.               */
+int flashd_attn_fwd(const void* q, const void* k, const void* v, void* o,
+                    int B, int H, int Nq, int Nk, int d, float scale, int causal,
+                    void* stream);
+
+/* Same computation with options.  in_dtype must be FLASHD_BF16.  out_dtype
+ * selects the type of o (FLASHD_BF16 or FLASHD_F32).  lse_out (nullable,
+ * [B,H,Nq] fp32) receives the final state L_N = s_N - ln w_N = ln sum_j e^{s_j}
+ * (natural log; Eq. w-basic solved for the running sum).                  */
+int flashd_attn_fwd_ex(const void* q, const void* k, const void* v, void* o, float* lse_out,
+                       int in_dtype, int out_dtype,
+                       int B, int H, int Nq, int Nk, int d, float scale, int causal,
+                       void* stream);
+
+/* ------------------------------------------------------------------------
+ * Per-key forward: Algorithm 3 exactly as stated, one key at a time, state
+ * (s_{i-1}, ln w_{i-1}, o_{i-1}) per query, w_1 = 1, weight by Eq. (w-last)
+ * with sigma evaluated over the full range (no clamp, no skip), blend in the
+ * one-multiplier form of Sec. IV-A, o + (v - o) w.  Scores and the carried
+ * ln w are kept in fp64, sigma / ln sigma / blend in fp32.
+ *
+ * flashd_attn_fwd_f32: fp32 in, fp32 out.
+ * flashd_attn_fwd_perkey: in_dtype / out_dtype in {FLASHD_BF16, FLASHD_F32}.
+ * d must be 32, 64, 128 or 256.  lse_out nullable.                        */
+int flashd_attn_fwd_f32(const void* q, const void* k, const void* v, void* o,
+                        int B, int H, int Nq, int Nk, int d, float scale, int causal,
+                        void* stream);
+int flashd_attn_fwd_perkey(const void* q, const void* k, const void* v, void* o, float* lse_out,
+                           int in_dtype, int out_dtype,
+                           int B, int H, int Nq, int Nk, int d, float scale, int causal,
+                           void* stream);
+
+/* ------------------------------------------------------------------------
+ * Split-K forward for long key sequences and few queries (decode).
+ * Non-causal, bf16 in, d = 128 or 64.
+ *
+ * The Nk keys are cut into num_splits contiguous ranges of
+ * ceil(Nk / num_splits) keys.  flashd_splitk_partial runs the tile form of
+ * Algorithm 3 over each range from an empty state and writes, per
+ * (b, h, query, split), the range's own attention output o_p (d floats)
+ * followed by its state L_p (1 float; -inf for an empty range) to
+ * `workspace`, laid out [B,H,Nq,num_splits,d+1] fp32.
+ * flashd_splitk_combine folds the partials in split order as super-keys
+ * (score L_p, value o_p) with Eq. (w-last) and the Sec. IV-A blend:
+ *     W = sigma(L_p - L_acc); o_acc += (o_p - o_acc) W; L_acc = L_p - ln W,
+ * the first non-empty split taking W = 1.  No division is made anywhere.
+ *
+ * workspace: device memory of at least flashd_splitk_workspace_bytes(...)
+ * bytes, 16-byte aligned, owned by the caller; contents need not be
+ * initialised.  num_splits in [1, FLASHD_MAX_SPLITS] and <= Nk.
+ * flashd_splitk_num_splits returns the split count the library would pick.
+ * flashd_attn_fwd_splitk queues partial + combine on `stream`
+ * (num_splits <= 0: library's choice; the workspace must then be sized for
+ * flashd_splitk_num_splits(...)).                                          */
+size_t flashd_splitk_workspace_bytes(int B, int H, int Nq, int d, int num_splits);
+int flashd_splitk_num_splits(int B, int H, int Nq, int Nk, int d);
+int flashd_splitk_partial(const void* q, const void* k, const void* v,
+                          void* workspace, size_t workspace_bytes,
+                          int B, int H, int Nq, int Nk, int d, float scale,
+                          int num_splits, void* stream);
+int flashd_splitk_combine(const void* workspace, void* o, float* lse_out,
+                          int B, int H, int Nq, int d, int num_splits, int out_dtype,
+                          void* stream);
+int flashd_attn_fwd_splitk(const void* q, const void* k, const void* v, void* o,
+                           void* workspace, size_t workspace_bytes,
+                           int B, int H, int Nq, int Nk, int d, float scale,
+                           int num_splits, void* stream);
+
+/* ------------------------------------------------------------------------
+ * End-to-end call on HOST buffers: q, k, v, o are host pointers (pinned
+ * memory gives asynchronous copies).  The call allocates device buffers from
+ * the stream-ordered pool of the current device, copies q, k, v in, runs the
+ * forward selected by `path`, copies o back, frees the buffers and
+ * SYNCHRONISES `stream` before returning.
+ * path 0: flashd_attn_fwd (bf16)   path 1: flashd_attn_fwd_f32
+ * path 2: flashd_attn_fwd_splitk (bf16, library's split count)            */
+int flashd_attn_fwd_host(const void* q, const void* k, const void* v, void* o,
+                         int path, int B, int H, int Nq, int Nk, int d, float scale,
+                         int causal, void* stream);
+
+/* ------------------------------------------------------------------------
+ * Utilities.
+ * flashd_last_device_status synchronises `stream`, then reads and clears the
+ * device-side status word of the current device: FLASHD_OK, or
+ * FLASHD_ERR_TIMEOUT if a bounded wait inside a kernel gave up (its output is
+ * then undefined).  detail (nullable, HOST int[4]) receives
+ * {code, blockIdx.x, which wait, iteration}.                              */
+int flashd_last_device_status(void* stream, int* detail);
+const char* flashd_status_string(int status);
+int flashd_version(void);
+/* Number of kernels launched by this library in this process so far. */
+long long flashd_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLASHD_H */

@@ -1,0 +1,240 @@
+"""ctypes binding with the same names as the C ABI in ``include/flashd.h``.
+
+Tensor arguments are torch tensors; the functions pass their ``data_ptr()`` and
+sizes through and raise :class:`FlashdError` on a non-zero status.  Outputs are
+allocated by the caller or, when omitted, with ``torch.empty`` on the inputs'
+device (torch is used for device memory and streams only).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import threading
+
+BF16, F32 = 0, 1
+MAX_SPLITS = 64
+
+EXPORTED_SYMBOLS = (
+    "flashd_attn_fwd", "flashd_attn_fwd_ex", "flashd_attn_fwd_f32", "flashd_attn_fwd_perkey",
+    "flashd_splitk_workspace_bytes", "flashd_splitk_num_splits", "flashd_splitk_partial",
+    "flashd_splitk_combine", "flashd_attn_fwd_splitk", "flashd_attn_fwd_host",
+    "flashd_last_device_status", "flashd_status_string", "flashd_version", "flashd_launch_count",
+)
+
+_lock = threading.Lock()
+_lib = None
+
+
+class FlashdError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: flashd status {status} ({status_string(status)})")
+
+
+def lib_path() -> str:
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "libflashd.so")
+
+
+def lib() -> ctypes.CDLL:
+    """Load ``libflashd.so``; raises if it has not been built (no fallback)."""
+    global _lib
+    with _lock:
+        if _lib is None:
+            path = lib_path()
+            if not os.path.exists(path):
+                raise FileNotFoundError(
+                    f"{path} is missing: build it with `python -m paper_2505_14201_b200.build` "
+                    "(nvcc, sm_100a). There is no CPU fallback.")
+            L = ctypes.CDLL(path)
+            vp, ci, cf, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+            fwd = [vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, ci, vp]
+            L.flashd_attn_fwd.argtypes = fwd
+            L.flashd_attn_fwd_f32.argtypes = fwd
+            ex = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, ci, vp]
+            L.flashd_attn_fwd_ex.argtypes = ex
+            L.flashd_attn_fwd_perkey.argtypes = ex
+            L.flashd_splitk_workspace_bytes.argtypes = [ci, ci, ci, ci, ci]
+            L.flashd_splitk_workspace_bytes.restype = sz
+            L.flashd_splitk_num_splits.argtypes = [ci, ci, ci, ci, ci]
+            L.flashd_splitk_partial.argtypes = [vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
+            L.flashd_splitk_combine.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, vp]
+            L.flashd_attn_fwd_splitk.argtypes = [vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
+            L.flashd_attn_fwd_host.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp]
+            L.flashd_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
+            L.flashd_status_string.argtypes = [ci]
+            L.flashd_status_string.restype = ctypes.c_char_p
+            L.flashd_version.argtypes = []
+            L.flashd_launch_count.argtypes = []
+            L.flashd_launch_count.restype = ctypes.c_longlong
+            _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().flashd_status_string(int(status)).decode()
+
+
+def version() -> int:
+    return int(lib().flashd_version())
+
+
+def launch_count() -> int:
+    return int(lib().flashd_launch_count())
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise FlashdError(int(status), where)
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        import torch
+        return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, int):
+        return ctypes.c_void_p(stream)
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _dims(q, k, v):
+    if q.dim() != 4 or k.dim() != 4 or v.dim() != 4:
+        raise ValueError("q, k, v must be [B, H, N, d]")
+    B, H, Nq, d = q.shape
+    Nk = k.shape[2]
+    if tuple(k.shape) != (B, H, Nk, d) or tuple(v.shape) != (B, H, Nk, d):
+        raise ValueError("shape mismatch between q, k, v")
+    if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous()):
+        raise ValueError("q, k, v must be contiguous")
+    return B, H, Nq, Nk, d
+
+
+def _dtype_code(t):
+    import torch
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float32:
+        return F32
+    raise ValueError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t):
+    return ctypes.c_void_p(0 if t is None else t.data_ptr())
+
+
+def flashd_attn_fwd(q, k, v, scale, causal=False, o=None, stream=None):
+    """bf16 tiled tensor-core forward; returns ``o`` ([B,H,Nq,d] bf16)."""
+    import torch
+    B, H, Nq, Nk, d = _dims(q, k, v)
+    if o is None:
+        o = torch.empty_like(q)
+    _check(lib().flashd_attn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, H, Nq, Nk, d,
+                                 float(scale), int(bool(causal)), _stream_ptr(stream)), "flashd_attn_fwd")
+    return o
+
+
+def flashd_attn_fwd_ex(q, k, v, scale, causal=False, out_dtype=None, return_lse=False, o=None,
+                       stream=None):
+    import torch
+    B, H, Nq, Nk, d = _dims(q, k, v)
+    out_dtype = q.dtype if out_dtype is None else out_dtype
+    if o is None:
+        o = torch.empty(q.shape, dtype=out_dtype, device=q.device)
+    lse = torch.empty((B, H, Nq), dtype=torch.float32, device=q.device) if return_lse else None
+    _check(lib().flashd_attn_fwd_ex(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _dtype_code(q),
+                                    _dtype_code(o), B, H, Nq, Nk, d, float(scale), int(bool(causal)),
+                                    _stream_ptr(stream)), "flashd_attn_fwd_ex")
+    return (o, lse) if return_lse else o
+
+
+def flashd_attn_fwd_f32(q, k, v, scale, causal=False, o=None, stream=None):
+    """fp32 per-key forward (Algorithm 3 one key at a time)."""
+    import torch
+    B, H, Nq, Nk, d = _dims(q, k, v)
+    if q.dtype != torch.float32:
+        raise ValueError("flashd_attn_fwd_f32 takes fp32 tensors")
+    if o is None:
+        o = torch.empty_like(q)
+    _check(lib().flashd_attn_fwd_f32(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, H, Nq, Nk, d,
+                                     float(scale), int(bool(causal)), _stream_ptr(stream)), "flashd_attn_fwd_f32")
+    return o
+
+
+def flashd_attn_fwd_perkey(q, k, v, scale, causal=False, out_dtype=None, return_lse=False, o=None,
+                           stream=None):
+    import torch
+    B, H, Nq, Nk, d = _dims(q, k, v)
+    out_dtype = q.dtype if out_dtype is None else out_dtype
+    if o is None:
+        o = torch.empty(q.shape, dtype=out_dtype, device=q.device)
+    lse = torch.empty((B, H, Nq), dtype=torch.float32, device=q.device) if return_lse else None
+    _check(lib().flashd_attn_fwd_perkey(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _dtype_code(q),
+                                        _dtype_code(o), B, H, Nq, Nk, d, float(scale), int(bool(causal)),
+                                        _stream_ptr(stream)), "flashd_attn_fwd_perkey")
+    return (o, lse) if return_lse else o
+
+
+def flashd_splitk_workspace_bytes(B, H, Nq, d, num_splits) -> int:
+    return int(lib().flashd_splitk_workspace_bytes(B, H, Nq, d, num_splits))
+
+
+def flashd_splitk_num_splits(B, H, Nq, Nk, d) -> int:
+    return int(lib().flashd_splitk_num_splits(B, H, Nq, Nk, d))
+
+
+def flashd_splitk_partial(q, k, v, scale, num_splits, workspace=None, stream=None):
+    """Returns the workspace tensor ``[B,H,Nq,num_splits,d+1]`` fp32 (o_p | L_p)."""
+    import torch
+    B, H, Nq, Nk, d = _dims(q, k, v)
+    if workspace is None:
+        workspace = torch.empty((B, H, Nq, num_splits, d + 1), dtype=torch.float32, device=q.device)
+    _check(lib().flashd_splitk_partial(_ptr(q), _ptr(k), _ptr(v), _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), B, H, Nq, Nk, d,
+                                       float(scale), int(num_splits), _stream_ptr(stream)), "flashd_splitk_partial")
+    return workspace
+
+
+def flashd_splitk_combine(workspace, B, H, Nq, d, num_splits, out_dtype=None, return_lse=False, o=None,
+                          stream=None):
+    import torch
+    out_dtype = torch.bfloat16 if out_dtype is None else out_dtype
+    if o is None:
+        o = torch.empty((B, H, Nq, d), dtype=out_dtype, device=workspace.device)
+    lse = torch.empty((B, H, Nq), dtype=torch.float32, device=workspace.device) if return_lse else None
+    _check(lib().flashd_splitk_combine(_ptr(workspace), _ptr(o), _ptr(lse), B, H, Nq, d, int(num_splits),
+                                       _dtype_code(o), _stream_ptr(stream)), "flashd_splitk_combine")
+    return (o, lse) if return_lse else o
+
+
+def flashd_attn_fwd_splitk(q, k, v, scale, num_splits=0, workspace=None, o=None, stream=None):
+    """Split-K forward (partial + combine); ``num_splits <= 0`` lets the library choose."""
+    import torch
+    B, H, Nq, Nk, d = _dims(q, k, v)
+    S = num_splits if num_splits > 0 else flashd_splitk_num_splits(B, H, Nq, Nk, d)
+    if workspace is None:
+        workspace = torch.empty((B, H, Nq, max(S, 1), d + 1), dtype=torch.float32, device=q.device)
+    if o is None:
+        o = torch.empty_like(q)
+    _check(lib().flashd_attn_fwd_splitk(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(workspace),
+                                        workspace.numel() * workspace.element_size(), B, H, Nq, Nk, d,
+                                        float(scale), int(num_splits), _stream_ptr(stream)), "flashd_attn_fwd_splitk")
+    return o
+
+
+def flashd_attn_fwd_host(q, k, v, scale, causal=False, path=0, o=None, stream=None):
+    """End-to-end call on HOST tensors (pinned for asynchronous copies); synchronises."""
+    import torch
+    if q.is_cuda or k.is_cuda or v.is_cuda:
+        raise ValueError("flashd_attn_fwd_host takes host tensors")
+    B, H, Nq, Nk, d = _dims(q, k, v)
+    if o is None:
+        o = torch.empty_like(q, pin_memory=True)
+    _check(lib().flashd_attn_fwd_host(_ptr(q), _ptr(k), _ptr(v), _ptr(o), int(path), B, H, Nq, Nk, d,
+                                      float(scale), int(bool(causal)), _stream_ptr(stream)), "flashd_attn_fwd_host")
+    return o
+
+
+def flashd_last_device_status(stream=None):
+    """(status, [code, block, which wait, iteration]) after synchronising the stream."""
+    detail = (ctypes.c_int * 4)()
+    st = lib().flashd_last_device_status(_stream_ptr(stream), detail)
+    return int(st), list(detail)

@@ -1,0 +1,347 @@
+// C ABI of the FLASH-D attention library (see include/flashd.h): argument
+// validation, tensor-map construction and kernel launches.  One translation
+// unit: the kernels are included as headers.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstdint>
+#include <mutex>
+
+#include "flashd.h"
+#include "flashd_common.cuh"
+#include "flashd_decode.cuh"
+#include "flashd_perkey.cuh"
+#include "flashd_prefill.cuh"
+
+namespace {
+
+using namespace flashd;
+
+std::atomic<long long> g_launches{0};
+
+inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_common(const void* q, const void* k, const void* v, const void* o, int B, int H, int Nq, int Nk,
+                 int d, float scale) {
+    if (!q || !k || !v || !o) return FLASHD_ERR_NULL;
+    if (B <= 0 || H <= 0 || Nq <= 0 || Nk <= 0 || d <= 0 || !std::isfinite(scale)) return FLASHD_ERR_SHAPE;
+    if ((long long)B * H > 0x7fffffffLL / 2) return FLASHD_ERR_SHAPE;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return FLASHD_ERR_ALIGN;
+    return FLASHD_OK;
+}
+
+int after_launch() {
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? FLASHD_OK : FLASHD_ERR_CUDA;
+}
+
+int sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+// ----------------------------------------------------------------- tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+// [BH, N, D] bf16 tensor, box = 64 columns x 128 rows x 1 head, 128-byte swizzle,
+// rows outside [0, N) read as zero.
+bool make_map(CUtensorMap* map, const void* base, int BH, int N, int D) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)N, (cuuint64_t)BH};
+    const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)N * D * 2};
+    const cuuint32_t box[3] = {64, 128, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D>
+int launch_prefill(const void* q, const void* k, const void* v, void* o, float* lse, int out_f32, int BH, int Nq,
+                   int Nk, float scale, int causal, cudaStream_t stream) {
+    using C = PrefillCfg<D>;
+    CUtensorMap mq, mk, mv;
+    if (!make_map(&mq, q, BH, Nq, D) || !make_map(&mk, k, BH, Nk, D) || !make_map(&mv, v, BH, Nk, D))
+        return FLASHD_ERR_CUDA;
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FLASHD_ERR_CUDA;
+    if (!attr_set[dev]) {
+        if (cudaFuncSetAttribute(prefill_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) !=
+            cudaSuccess)
+            return FLASHD_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    PrefillParams prm;
+    prm.o = o;
+    prm.lse = lse;
+    prm.BH = BH;
+    prm.Nq = Nq;
+    prm.Nk = Nk;
+    prm.scale_log2e = scale * kLog2e;
+    prm.causal = causal ? 1 : 0;
+    prm.out_f32 = out_f32;
+    prm.n_qpairs = (Nq + 255) / 256;
+    prm.n_work = BH * prm.n_qpairs;
+    const int sms = sm_count();
+    if (sms <= 0) return FLASHD_ERR_CUDA;
+    const int grid = prm.n_work < sms ? prm.n_work : sms;
+    prefill_kernel<D><<<grid, C::kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, prm);
+    return after_launch();
+}
+
+template <typename TIn, typename TOut>
+int launch_perkey_t(const void* q, const void* k, const void* v, void* o, float* lse, long long rows, int Nq,
+                    int Nk, int d, float scale, int causal, cudaStream_t stream) {
+    const int warps = 4;
+    const long long blocks = (rows + warps - 1) / warps;
+    if (blocks > 0x7fffffffLL) return FLASHD_ERR_SHAPE;
+    const TIn* qq = static_cast<const TIn*>(q);
+    const TIn* kk = static_cast<const TIn*>(k);
+    const TIn* vv = static_cast<const TIn*>(v);
+    TOut* oo = static_cast<TOut*>(o);
+    switch (d) {
+        case 32: perkey_kernel<TIn, TOut, 1><<<(unsigned)blocks, warps * 32, 0, stream>>>(qq, kk, vv, oo, lse, rows, Nq, Nk, scale, causal); break;
+        case 64: perkey_kernel<TIn, TOut, 2><<<(unsigned)blocks, warps * 32, 0, stream>>>(qq, kk, vv, oo, lse, rows, Nq, Nk, scale, causal); break;
+        case 128: perkey_kernel<TIn, TOut, 4><<<(unsigned)blocks, warps * 32, 0, stream>>>(qq, kk, vv, oo, lse, rows, Nq, Nk, scale, causal); break;
+        case 256: perkey_kernel<TIn, TOut, 8><<<(unsigned)blocks, warps * 32, 0, stream>>>(qq, kk, vv, oo, lse, rows, Nq, Nk, scale, causal); break;
+        default: return FLASHD_ERR_UNSUPPORTED;
+    }
+    return after_launch();
+}
+
+template <int D>
+int launch_partial(const void* q, const void* k, const void* v, void* ws, long long rows, int Nq, int Nk,
+                   float scale, int num_splits, cudaStream_t stream) {
+    using C = DecodeCfg<D>;
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FLASHD_ERR_CUDA;
+    if (!attr_set[dev]) {
+        if (cudaFuncSetAttribute(splitk_partial_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 C::kSmemBytes) != cudaSuccess)
+            return FLASHD_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    const int sms = sm_count();
+    if (sms <= 0) return FLASHD_ERR_CUDA;
+    const long long items = rows * num_splits;
+    const int grid = (int)(items < sms ? items : sms);
+    splitk_partial_kernel<D><<<grid, C::kThreads, C::kSmemBytes, stream>>>(
+        static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
+        static_cast<const __nv_bfloat16*>(v), static_cast<float*>(ws), rows, Nq, Nk, scale * kLog2e, num_splits);
+    return after_launch();
+}
+
+int check_splits(int Nk, int num_splits) {
+    if (num_splits < 1 || num_splits > FLASHD_MAX_SPLITS || num_splits > Nk) return FLASHD_ERR_WORKSPACE;
+    // every split but the last must be non-empty by construction; the last one is
+    // non-empty iff (S-1)*ceil(Nk/S) < Nk, otherwise it is written as empty (L = -inf)
+    return FLASHD_OK;
+}
+
+}  // namespace
+
+// ============================================================================ C ABI
+extern "C" {
+
+int flashd_version(void) { return 100; }
+
+long long flashd_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* flashd_status_string(int status) {
+    switch (status) {
+        case FLASHD_OK: return "ok";
+        case FLASHD_ERR_NULL: return "null pointer";
+        case FLASHD_ERR_SHAPE: return "invalid size or scale";
+        case FLASHD_ERR_UNSUPPORTED: return "unsupported head size, dtype or mode";
+        case FLASHD_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case FLASHD_ERR_WORKSPACE: return "workspace too small or bad split count";
+        case FLASHD_ERR_CUDA: return "CUDA call failed";
+        case FLASHD_ERR_TIMEOUT: return "bounded wait inside a kernel ran out";
+        default: return "unknown status";
+    }
+}
+
+int flashd_attn_fwd_ex(const void* q, const void* k, const void* v, void* o, float* lse_out, int in_dtype,
+                       int out_dtype, int B, int H, int Nq, int Nk, int d, float scale, int causal, void* stream) {
+    const int st = check_common(q, k, v, o, B, H, Nq, Nk, d, scale);
+    if (st != FLASHD_OK) return st;
+    if (in_dtype != FLASHD_BF16 || (out_dtype != FLASHD_BF16 && out_dtype != FLASHD_F32)) return FLASHD_ERR_UNSUPPORTED;
+    if (scale == 0.f) return FLASHD_ERR_UNSUPPORTED;
+    if (o == q || o == k || o == v) return FLASHD_ERR_SHAPE;
+    const int BH = B * H;
+    if (d == 128) return launch_prefill<128>(q, k, v, o, lse_out, out_dtype == FLASHD_F32, BH, Nq, Nk, scale, causal, as_stream(stream));
+    if (d == 64) return launch_prefill<64>(q, k, v, o, lse_out, out_dtype == FLASHD_F32, BH, Nq, Nk, scale, causal, as_stream(stream));
+    return FLASHD_ERR_UNSUPPORTED;
+}
+
+int flashd_attn_fwd(const void* q, const void* k, const void* v, void* o, int B, int H, int Nq, int Nk, int d,
+                    float scale, int causal, void* stream) {
+    return flashd_attn_fwd_ex(q, k, v, o, nullptr, FLASHD_BF16, FLASHD_BF16, B, H, Nq, Nk, d, scale, causal, stream);
+}
+
+int flashd_attn_fwd_perkey(const void* q, const void* k, const void* v, void* o, float* lse_out, int in_dtype,
+                           int out_dtype, int B, int H, int Nq, int Nk, int d, float scale, int causal,
+                           void* stream) {
+    const int st = check_common(q, k, v, o, B, H, Nq, Nk, d, scale);
+    if (st != FLASHD_OK) return st;
+    if (d != 32 && d != 64 && d != 128 && d != 256) return FLASHD_ERR_UNSUPPORTED;
+    const long long rows = (long long)B * H * Nq;
+    cudaStream_t s = as_stream(stream);
+    if (in_dtype == FLASHD_F32 && out_dtype == FLASHD_F32)
+        return launch_perkey_t<float, float>(q, k, v, o, lse_out, rows, Nq, Nk, d, scale, causal, s);
+    if (in_dtype == FLASHD_BF16 && out_dtype == FLASHD_BF16)
+        return launch_perkey_t<__nv_bfloat16, __nv_bfloat16>(q, k, v, o, lse_out, rows, Nq, Nk, d, scale, causal, s);
+    if (in_dtype == FLASHD_BF16 && out_dtype == FLASHD_F32)
+        return launch_perkey_t<__nv_bfloat16, float>(q, k, v, o, lse_out, rows, Nq, Nk, d, scale, causal, s);
+    return FLASHD_ERR_UNSUPPORTED;
+}
+
+int flashd_attn_fwd_f32(const void* q, const void* k, const void* v, void* o, int B, int H, int Nq, int Nk, int d,
+                        float scale, int causal, void* stream) {
+    return flashd_attn_fwd_perkey(q, k, v, o, nullptr, FLASHD_F32, FLASHD_F32, B, H, Nq, Nk, d, scale, causal, stream);
+}
+
+size_t flashd_splitk_workspace_bytes(int B, int H, int Nq, int d, int num_splits) {
+    if (B <= 0 || H <= 0 || Nq <= 0 || d <= 0 || num_splits <= 0) return 0;
+    return (size_t)B * H * Nq * num_splits * (size_t)(d + 1) * sizeof(float);
+}
+
+int flashd_splitk_num_splits(int B, int H, int Nq, int Nk, int d) {
+    (void)d;
+    if (B <= 0 || H <= 0 || Nq <= 0 || Nk <= 0) return 0;
+    const long long rows = (long long)B * H * Nq;
+    // enough work items for ~32 waves on a 148-SM part, splits of at least 512 keys
+    long long want = (32LL * 148 + rows - 1) / rows;
+    int s = 1;
+    while (s < want && s < FLASHD_MAX_SPLITS) s *= 2;
+    if (Nk >= 8192 && s < 2) s = 2;
+    while (s > 1 && Nk / s < 512) s /= 2;
+    return s;
+}
+
+int flashd_splitk_partial(const void* q, const void* k, const void* v, void* workspace, size_t workspace_bytes,
+                          int B, int H, int Nq, int Nk, int d, float scale, int num_splits, void* stream) {
+    const int st = check_common(q, k, v, workspace, B, H, Nq, Nk, d, scale);
+    if (st != FLASHD_OK) return st;
+    if (d != 128 && d != 64) return FLASHD_ERR_UNSUPPORTED;
+    const int cs = check_splits(Nk, num_splits);
+    if (cs != FLASHD_OK) return cs;
+    if (workspace_bytes < flashd_splitk_workspace_bytes(B, H, Nq, d, num_splits)) return FLASHD_ERR_WORKSPACE;
+    const long long rows = (long long)B * H * Nq;
+    if (d == 128) return launch_partial<128>(q, k, v, workspace, rows, Nq, Nk, scale, num_splits, as_stream(stream));
+    return launch_partial<64>(q, k, v, workspace, rows, Nq, Nk, scale, num_splits, as_stream(stream));
+}
+
+int flashd_splitk_combine(const void* workspace, void* o, float* lse_out, int B, int H, int Nq, int d,
+                          int num_splits, int out_dtype, void* stream) {
+    if (!workspace || !o) return FLASHD_ERR_NULL;
+    if (B <= 0 || H <= 0 || Nq <= 0 || d <= 0) return FLASHD_ERR_SHAPE;
+    if (d != 128 && d != 64) return FLASHD_ERR_UNSUPPORTED;
+    if (out_dtype != FLASHD_BF16 && out_dtype != FLASHD_F32) return FLASHD_ERR_UNSUPPORTED;
+    if (num_splits < 1 || num_splits > FLASHD_MAX_SPLITS) return FLASHD_ERR_WORKSPACE;
+    if (!aligned16(workspace) || !aligned16(o)) return FLASHD_ERR_ALIGN;
+    const long long rows = (long long)B * H * Nq;
+    if (rows > 0x7fffffffLL) return FLASHD_ERR_SHAPE;
+    const float* ws = static_cast<const float*>(workspace);
+    cudaStream_t s = as_stream(stream);
+    if (d == 128) {
+        if (out_dtype == FLASHD_F32) splitk_combine_kernel<128, float><<<(unsigned)rows, 128, 0, s>>>(ws, static_cast<float*>(o), lse_out, num_splits);
+        else splitk_combine_kernel<128, __nv_bfloat16><<<(unsigned)rows, 128, 0, s>>>(ws, static_cast<__nv_bfloat16*>(o), lse_out, num_splits);
+    } else {
+        if (out_dtype == FLASHD_F32) splitk_combine_kernel<64, float><<<(unsigned)rows, 64, 0, s>>>(ws, static_cast<float*>(o), lse_out, num_splits);
+        else splitk_combine_kernel<64, __nv_bfloat16><<<(unsigned)rows, 64, 0, s>>>(ws, static_cast<__nv_bfloat16*>(o), lse_out, num_splits);
+    }
+    return after_launch();
+}
+
+int flashd_attn_fwd_splitk(const void* q, const void* k, const void* v, void* o, void* workspace,
+                           size_t workspace_bytes, int B, int H, int Nq, int Nk, int d, float scale, int num_splits,
+                           void* stream) {
+    if (!o) return FLASHD_ERR_NULL;
+    if (num_splits <= 0) num_splits = flashd_splitk_num_splits(B, H, Nq, Nk, d);
+    if (!workspace) return FLASHD_ERR_NULL;
+    int st = flashd_splitk_partial(q, k, v, workspace, workspace_bytes, B, H, Nq, Nk, d, scale, num_splits, stream);
+    if (st != FLASHD_OK) return st;
+    return flashd_splitk_combine(workspace, o, nullptr, B, H, Nq, d, num_splits, FLASHD_BF16, stream);
+}
+
+int flashd_attn_fwd_host(const void* q, const void* k, const void* v, void* o, int path, int B, int H, int Nq,
+                         int Nk, int d, float scale, int causal, void* stream) {
+    if (!q || !k || !v || !o) return FLASHD_ERR_NULL;
+    if (B <= 0 || H <= 0 || Nq <= 0 || Nk <= 0 || d <= 0 || !std::isfinite(scale)) return FLASHD_ERR_SHAPE;
+    if (path < 0 || path > 2) return FLASHD_ERR_UNSUPPORTED;
+    if (path == 2 && causal) return FLASHD_ERR_UNSUPPORTED;
+    const size_t esz = (path == 1) ? 4 : 2;
+    const size_t qb = (size_t)B * H * Nq * d * esz, kb = (size_t)B * H * Nk * d * esz;
+    cudaStream_t s = as_stream(stream);
+    int splits = 0;
+    size_t wsb = 0;
+    if (path == 2) {
+        splits = flashd_splitk_num_splits(B, H, Nq, Nk, d);
+        wsb = flashd_splitk_workspace_bytes(B, H, Nq, d, splits);
+    }
+    void *dq = nullptr, *dk = nullptr, *dv = nullptr, *dout = nullptr, *dws = nullptr;
+    int st = FLASHD_OK;
+    bool ok = cudaMallocAsync(&dq, qb, s) == cudaSuccess && cudaMallocAsync(&dk, kb, s) == cudaSuccess &&
+              cudaMallocAsync(&dv, kb, s) == cudaSuccess && cudaMallocAsync(&dout, qb, s) == cudaSuccess &&
+              (wsb == 0 || cudaMallocAsync(&dws, wsb, s) == cudaSuccess);
+    ok = ok && cudaMemcpyAsync(dq, q, qb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
+         cudaMemcpyAsync(dk, k, kb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
+         cudaMemcpyAsync(dv, v, kb, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (!ok) st = FLASHD_ERR_CUDA;
+    if (st == FLASHD_OK) {
+        if (path == 0) st = flashd_attn_fwd(dq, dk, dv, dout, B, H, Nq, Nk, d, scale, causal, stream);
+        else if (path == 1) st = flashd_attn_fwd_f32(dq, dk, dv, dout, B, H, Nq, Nk, d, scale, causal, stream);
+        else st = flashd_attn_fwd_splitk(dq, dk, dv, dout, dws, wsb, B, H, Nq, Nk, d, scale, splits, stream);
+    }
+    if (st == FLASHD_OK && cudaMemcpyAsync(o, dout, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) st = FLASHD_ERR_CUDA;
+    if (dq) cudaFreeAsync(dq, s);
+    if (dk) cudaFreeAsync(dk, s);
+    if (dv) cudaFreeAsync(dv, s);
+    if (dout) cudaFreeAsync(dout, s);
+    if (dws) cudaFreeAsync(dws, s);
+    if (cudaStreamSynchronize(s) != cudaSuccess && st == FLASHD_OK) st = FLASHD_ERR_CUDA;
+    return st;
+}
+
+int flashd_last_device_status(void* stream, int* detail) {
+    if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return FLASHD_ERR_CUDA;
+    unsigned int h[4] = {0, 0, 0, 0};
+    if (cudaMemcpyFromSymbol(h, flashd::g_status, sizeof(h)) != cudaSuccess) return FLASHD_ERR_CUDA;
+    if (h[0] != 0) {
+        const unsigned int z[4] = {0, 0, 0, 0};
+        cudaMemcpyToSymbol(flashd::g_status, z, sizeof(z));
+    }
+    if (detail) for (int i = 0; i < 4; ++i) detail[i] = (int)h[i];
+    return (int)h[0];
+}
+
+}  // extern "C"

@@ -1,0 +1,250 @@
+// Split-K FLASH-D forward for long key sequences (decode) and its combine.
+//
+// Partial kernel: one work item = (query row, split).  A producer warp streams
+// the split's K and V rows from HBM into a shared-memory ring with bulk async
+// copies; eight consumer warps fold them into G independent running states
+// (L, o) - one per group of lanes that covers a key row - using the group form
+// of Algorithm 3: for a group of keys with scores s_j and log-sum-exp L_T,
+//     W = sigma(L_T - L_old)                       Eq. (w-last) on the super-key
+//     L_new = L_T - ln W,  P_j = exp(s_j - L_new),  alpha = exp(L_old - L_new)
+//     o <- alpha o + sum_j P_j v_j                  Eq. (out-final) for the group
+// so o is normalised after every group and nothing is divided at the end.  The
+// G states of the CTA are then merged, and later the splits are merged, by the
+// same super-key step in the one-multiplier form of Sec. IV-A:
+//     o <- o + (o_p - o) W,  L <- L_p - ln W.
+// L is kept in log2 units inside the kernels and written in natural log.
+#pragma once
+
+#include "flashd_common.cuh"
+
+namespace flashd {
+
+template <int D>
+struct DecodeCfg {
+    static constexpr int kChunk = 8192 / D;                  // keys per ring stage (16 KB of K, 16 KB of V)
+    static constexpr int kStages = 5;
+    static constexpr int kConsumerWarps = 8;
+    static constexpr int kThreads = (kConsumerWarps + 1) * 32;
+    static constexpr int kLanesPerRow = D / 8;               // 16-byte slices per key row
+    static constexpr int kRowsPerWarp = 32 / kLanesPerRow;
+    static constexpr int kGroups = kConsumerWarps * kRowsPerWarp;
+    static constexpr int kKeysPerGroup = kChunk / kGroups;   // = 4
+    static constexpr int kTileBytes = kChunk * D * 2;
+    static constexpr int kStageBytes = 2 * kTileBytes;
+    static constexpr int kMergeFloats = kGroups * (D + 1);
+    static constexpr int kSmemBytes = kStages * kStageBytes + kMergeFloats * 4 + 256;
+};
+
+// which-wait codes reported on timeout
+enum { kWaitDecFull = 0x100, kWaitDecEmpty = 0x101, kWaitDecMergeReady = 0x102, kWaitDecMergeFree = 0x103 };
+
+// One super-key step on (L_acc, W): returns W for merging a state with
+// log-sum-exp Lp (log2 units) into L_acc and updates L_acc.  sigma and
+// ln sigma are evaluated in their overflow-free branch form.
+__device__ __forceinline__ float superkey_weight(float& L_acc, float Lp) {
+    if (Lp == -INFINITY) return 0.f;                 // empty group: nothing to blend
+    if (L_acc == -INFINITY) { L_acc = Lp; return 1.f; }   // first group: W = 1 (Alg. 3, i = 1)
+    float W;
+    if (Lp >= L_acc) {
+        const float e = ex2(L_acc - Lp);
+        W = rcp(1.f + e);
+        L_acc = Lp + lg2(1.f + e);
+    } else {
+        const float e = ex2(Lp - L_acc);
+        W = e * rcp(1.f + e);
+        L_acc = L_acc + lg2(1.f + e);
+    }
+    return W;
+}
+
+template <int D>
+__global__ void __launch_bounds__(DecodeCfg<D>::kThreads, 1)
+splitk_partial_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                      const __nv_bfloat16* __restrict__ v, float* __restrict__ workspace,
+                      long long rows, int Nq, int Nk, float scale_log2e, int num_splits) {
+    using C = DecodeCfg<D>;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    unsigned char* ring = smem_raw;
+    float* merge = reinterpret_cast<float*>(smem_raw + C::kStages * C::kStageBytes);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + C::kStages * C::kStageBytes + C::kMergeFloats * 4);
+    uint64_t* full = bars;                   // [kStages]
+    uint64_t* empty = bars + C::kStages;     // [kStages]
+    uint64_t* merge_ready = bars + 2 * C::kStages;
+    uint64_t* merge_free = merge_ready + 1;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], C::kConsumerWarps); }
+        mbar_init(merge_ready, C::kConsumerWarps);
+        mbar_init(merge_free, C::kConsumerWarps);
+        mbar_init_fence();
+    }
+    __syncthreads();
+
+    const long long n_items = rows * num_splits;
+    const int per_split = (Nk + num_splits - 1) / num_splits;
+
+    if (warp == C::kConsumerWarps) {
+        // ------------------------------------------------------ producer
+        if (lane != 0) return;
+        uint32_t it = 0;
+        for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+            const long long row = item / num_splits;
+            const int split = (int)(item - row * num_splits);
+            const long long bh = row / Nq;
+            const int k0 = split * per_split;
+            const int k1 = min(k0 + per_split, Nk);
+            const __nv_bfloat16* kb = k + (bh * Nk) * (long long)D;
+            const __nv_bfloat16* vb = v + (bh * Nk) * (long long)D;
+            for (int c0 = k0; c0 < k1; c0 += C::kChunk, ++it) {
+                const int stage = it % C::kStages;
+                const uint32_t round = it / C::kStages;
+                if (round > 0 && !mbar_wait(&empty[stage], (round - 1) & 1, kWaitDecEmpty)) return;
+                const int nk = min(C::kChunk, k1 - c0);
+                const uint32_t bytes = (uint32_t)nk * D * 2;
+                unsigned char* dst = ring + stage * C::kStageBytes;
+                mbar_arrive_expect_tx(&full[stage], 2 * bytes);
+                bulk_load(dst, kb + (long long)c0 * D, bytes, &full[stage]);
+                bulk_load(dst + C::kTileBytes, vb + (long long)c0 * D, bytes, &full[stage]);
+            }
+        }
+        return;
+    }
+
+    // ---------------------------------------------------------- consumers
+    const int sl = lane % C::kLanesPerRow;                      // 16-byte slice of the row
+    const int g = warp * C::kRowsPerWarp + lane / C::kLanesPerRow;   // this lane's group
+    uint32_t it = 0;
+    uint32_t item_idx = 0;
+    for (long long item = blockIdx.x; item < n_items; item += gridDim.x, ++item_idx) {
+        const long long row = item / num_splits;
+        const int split = (int)(item - row * num_splits);
+        const int k0 = split * per_split;
+        const int k1 = min(k0 + per_split, Nk);
+
+        float qf[8];
+        {
+            const uint4 qw = *reinterpret_cast<const uint4*>(q + row * D + sl * 8);
+            const uint32_t w[4] = {qw.x, qw.y, qw.z, qw.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                qf[2 * e] = bf16_lo(w[e]) * scale_log2e;
+                qf[2 * e + 1] = bf16_hi(w[e]) * scale_log2e;
+            }
+        }
+        float of[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) of[e] = 0.f;
+        float L = -INFINITY;
+
+        for (int c0 = k0; c0 < k1; c0 += C::kChunk, ++it) {
+            const int stage = it % C::kStages;
+            const uint32_t round = it / C::kStages;
+            if (!mbar_wait(&full[stage], round & 1, kWaitDecFull)) return;
+            const int nk = min(C::kChunk, k1 - c0);
+            const unsigned char* ks = ring + stage * C::kStageBytes;
+            const unsigned char* vs = ks + C::kTileBytes;
+
+            float s[C::kKeysPerGroup];
+            bool valid[C::kKeysPerGroup];
+#pragma unroll
+            for (int m = 0; m < C::kKeysPerGroup; ++m) {
+                const int r = g + C::kGroups * m;
+                valid[m] = r < nk;
+                const uint4 kw = *reinterpret_cast<const uint4*>(ks + (r * D + sl * 8) * 2);
+                const uint32_t w[4] = {kw.x, kw.y, kw.z, kw.w};
+                float acc = 0.f;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    acc = fmaf(qf[2 * e], bf16_lo(w[e]), acc);
+                    acc = fmaf(qf[2 * e + 1], bf16_hi(w[e]), acc);
+                }
+                s[m] = acc;
+            }
+#pragma unroll
+            for (int sh = C::kLanesPerRow / 2; sh >= 1; sh >>= 1) {
+#pragma unroll
+                for (int m = 0; m < C::kKeysPerGroup; ++m) s[m] += __shfl_xor_sync(0xffffffffu, s[m], sh);
+            }
+            float ref = L;
+#pragma unroll
+            for (int m = 0; m < C::kKeysPerGroup; ++m) {
+                s[m] = valid[m] ? s[m] : -INFINITY;
+                ref = fmaxf(ref, s[m]);
+            }
+            if (ref != -INFINITY) {      // uniform within the group
+                // log-sum-exp of {L_old, s_j} relative to a group-local reference
+                const float e_old = ex2(L - ref);
+                float p[C::kKeysPerGroup];
+                float l = e_old;
+#pragma unroll
+                for (int m = 0; m < C::kKeysPerGroup; ++m) { p[m] = ex2(s[m] - ref); l += p[m]; }
+                const float inv = rcp(l);
+                const float alpha = e_old * inv;          // = 1 - W = exp(L_old - L_new)
+                L = ref + lg2(l);                          // L_new
+#pragma unroll
+                for (int e = 0; e < 8; ++e) of[e] *= alpha;
+#pragma unroll
+                for (int m = 0; m < C::kKeysPerGroup; ++m) {
+                    const int r = g + C::kGroups * m;
+                    const float P = p[m] * inv;            // = exp(s_j - L_new)
+                    uint4 vw = *reinterpret_cast<const uint4*>(vs + (r * D + sl * 8) * 2);
+                    if (!valid[m]) vw = make_uint4(0u, 0u, 0u, 0u);
+                    const uint32_t w[4] = {vw.x, vw.y, vw.z, vw.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        of[2 * e] = fmaf(P, bf16_lo(w[e]), of[2 * e]);
+                        of[2 * e + 1] = fmaf(P, bf16_hi(w[e]), of[2 * e + 1]);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty[stage]);
+        }
+
+        // ---- merge the CTA's group states, in group order, as super-keys
+        if (item_idx > 0 && !mbar_wait(merge_free, (item_idx - 1) & 1, kWaitDecMergeFree)) return;
+        {
+            float* mine = merge + g * (D + 1);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) mine[sl * 8 + e] = of[e];
+            if (sl == 0) mine[D] = L;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(merge_ready);
+        if (!mbar_wait(merge_ready, item_idx & 1, kWaitDecMergeReady)) return;
+        if (threadIdx.x < D) {
+            const int c = threadIdx.x;
+            float L_acc = -INFINITY, o_acc = 0.f;
+            for (int gg = 0; gg < C::kGroups; ++gg) {
+                const float W = superkey_weight(L_acc, merge[gg * (D + 1) + D]);
+                o_acc = fmaf(merge[gg * (D + 1) + c] - o_acc, W, o_acc);
+            }
+            float* wp = workspace + (row * num_splits + split) * (long long)(D + 1);
+            wp[c] = o_acc;
+            if (c == 0) wp[D] = L_acc * kLn2;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(merge_free);
+    }
+}
+
+// Combine: one CTA of D threads per query row; thread c owns output column c.
+template <int D, typename TOut>
+__global__ void __launch_bounds__(D)
+splitk_combine_kernel(const float* __restrict__ workspace, TOut* __restrict__ o,
+                      float* __restrict__ lse, int num_splits) {
+    const long long row = blockIdx.x;
+    const int c = threadIdx.x;
+    const float* wp = workspace + row * num_splits * (long long)(D + 1);
+    float L_acc = -INFINITY, o_acc = 0.f;
+    for (int s = 0; s < num_splits; ++s) {
+        const float W = superkey_weight(L_acc, wp[s * (D + 1) + D] * kLog2e);
+        o_acc = fmaf(wp[s * (D + 1) + c] - o_acc, W, o_acc);
+    }
+    o[row * D + c] = from_f32<TOut>(o_acc);
+    if (lse != nullptr && c == 0) lse[row] = L_acc * kLn2;
+}
+
+}  // namespace flashd

@@ -1,0 +1,508 @@
+// Tiled FLASH-D forward on the 5th-generation tensor cores (sm_100a).
+//
+// One CTA owns a pair of 128-row query tiles of one head and walks the key
+// sequence in tiles of 128 keys.  Per query tile and key tile:
+//   S = Q K^T                      tcgen05.mma, operands in shared memory (TMA),
+//                                  accumulator in tensor memory
+//   per row (one thread per row), with c = scale*log2(e) and L in log2 units:
+//       ref   = max(L_old, max_j c*s_j)          tile-local reference, not carried
+//       pt_j  = 2^(c*s_j - ref),  l = 2^(L_old - ref) + sum_j pt_j
+//       L_new = ref + log2 l                      = log-sum-exp of {L_old, s_j}
+//       P_j   = pt_j / l = exp(s_j - L_new)       weights of the tile's keys
+//       alpha = 2^(L_old - ref) / l = exp(L_old - L_new) = 1 - sum_j P_j
+//   O <- alpha O + P V             rescale by the correction warps, then
+//                                  tcgen05.mma with P read from tensor memory
+// This is Algorithm 3 of the paper applied to the tile as one super-key of score
+// L_T = log-sum-exp(s_j): Eq. (w-last) gives W = sigma(L_T - L_old), and
+// multiplying Eq. (out-final) through gives alpha = 1 - W and P_j = W exp(s_j - L_T).
+// O is normalised after every tile, the only carried state per row is L
+// (= s_i - ln w_i), there is no running maximum and no final division: the single
+// reciprocal 1/l per row and tile is the division hidden in the sigmoid.
+//
+// Warp roles (16 warps): 0-3 softmax of query tile 0, 4-7 softmax of query tile 1,
+// 8-11 correction + epilogue, 12 MMA issue, 13 TMA loads, 14-15 idle.
+// Tensor memory (512 columns): S0 | S1 | O0 | O1; P_i overlays the first 64
+// columns of S_i as packed bf16 pairs.
+// Every mbarrier wait is bounded; a wait that runs out records itself in the
+// device status word, raises the CTA's abort flag and the CTA drains and exits.
+#pragma once
+
+#include <cuda.h>
+
+#include "flashd_common.cuh"
+
+namespace flashd {
+
+template <int D>
+struct PrefillCfg {
+    static constexpr int kBlockM = 128;
+    static constexpr int kBlockN = 128;
+    static constexpr int kPanels = D / 64;                       // 64-column (128-byte) swizzle panels
+    static constexpr int kPanelBytes = 128 * 128;                // 128 rows x 128 bytes
+    static constexpr int kTileBytes = kPanels * kPanelBytes;     // one Q / K / V tile
+    static constexpr int kStages = (D == 128) ? 4 : 6;           // K/V ring
+    static constexpr int kThreads = 512;
+    static constexpr int kBarriers = 16 + 2 * kStages;
+    static constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + 2 * 128 * 4 + kBarriers * 8 + 64 + 1024;
+    static constexpr uint32_t kTmemCols = 512;
+    static constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO0 = 256, kColO1 = 256 + D;
+};
+
+enum {
+    kWaitQFull = 0x200, kWaitQEmpty, kWaitKVFull, kWaitKVEmpty, kWaitSFull, kWaitPFull,
+    kWaitAlphaFull, kWaitAlphaEmpty, kWaitPVDone, kWaitOReady
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* map, int c0, int c1, int c2,
+                                            uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(smem_dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t* smem_result, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
+                 "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 consecutive 32-bit columns of this thread's tensor-memory lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
+          "r"(taddr)
+        : "memory");
+}
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  lbo / sbo in bytes.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, A K-major, B K-major (b_mn = 0) or MN-major (1).
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N, int b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(N >> 3) << 17) |
+           ((uint32_t)(M >> 4) << 24);
+}
+
+struct PrefillParams {
+    void* o;            // [B*H, Nq, D] bf16 or fp32
+    float* lse;         // nullable, [B*H, Nq]
+    int BH, Nq, Nk;
+    float scale_log2e;  // scale * log2(e)
+    int causal;
+    int out_f32;
+    int n_qpairs;       // ceil(Nq / 256)
+    int n_work;         // BH * n_qpairs
+};
+
+// Wait bounded by an iteration count; also leaves when another thread of the
+// CTA has raised the abort flag.
+__device__ __forceinline__ bool pf_wait(uint64_t* bar, uint32_t parity, unsigned int which,
+                                        volatile uint32_t* abort_flag) {
+    for (uint32_t it = 0; it < kSpinFast; ++it)
+        if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_ns();
+    uint32_t it = 0;
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        __nanosleep(64);
+        if ((++it & 63u) == 0 && global_ns() - t0 > kWaitLimitNs) break;
+    }
+    report_timeout(which, parity);
+    *abort_flag = 1;
+    return false;
+}
+
+template <int D>
+__global__ void __launch_bounds__(512, 1)
+prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+               const __grid_constant__ CUtensorMap map_v, const PrefillParams prm) {
+    using C = PrefillCfg<D>;
+    extern __shared__ unsigned char smem_raw[];
+    // 1024-byte alignment for the swizzled tiles
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    unsigned char* sQ = smem;                               // 2 tiles
+    unsigned char* sKV = smem + 2 * C::kTileBytes;          // kStages tiles
+    float* sAlpha = reinterpret_cast<float*>(sKV + C::kStages * C::kTileBytes);   // [2][128]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sAlpha + 256);
+    uint64_t* q_full = bars;            // [2]
+    uint64_t* q_empty = bars + 2;       // [2]
+    uint64_t* s_full = bars + 4;        // [2]
+    uint64_t* p_full = bars + 6;        // [2]
+    uint64_t* alpha_full = bars + 8;    // [2]
+    uint64_t* alpha_empty = bars + 10;  // [2]
+    uint64_t* pv_done = bars + 12;      // [2]
+    uint64_t* o_ready = bars + 14;      // [2]
+    uint64_t* kv_full = bars + 16;                 // [kStages]
+    uint64_t* kv_empty = bars + 16 + C::kStages;   // [kStages]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::kBarriers);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&q_full[i], 1);
+            mbar_init(&q_empty[i], 1);
+            mbar_init(&s_full[i], 1);
+            mbar_init(&p_full[i], 128);
+            mbar_init(&alpha_full[i], 128);
+            mbar_init(&alpha_empty[i], 128);
+            mbar_init(&pv_done[i], 1);
+            mbar_init(&o_ready[i], 128);
+        }
+        for (int s = 0; s < C::kStages; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
+        *abort_flag = 0;
+        mbar_init_fence();
+    }
+    if (warp == 0) {
+        tmem_alloc(tmem_slot, C::kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int Nq = prm.Nq, Nk = prm.Nk;
+    const int n_kt_all = (Nk + 127) >> 7;
+    // key tiles needed by query tile i (rows q0 .. q0+127) of a work item; 0 if the tile is empty
+    auto n_tiles = [&](int q0) -> int {
+        if (q0 >= Nq) return 0;
+        if (!prm.causal) return n_kt_all;
+        const int lim = min(Nk, q0 + 128);
+        return (lim + 127) >> 7;
+    };
+
+    if (warp == 13) {
+        // ================================================================ TMA loader
+        reg_dec<48>();
+        if (lane == 0) {
+            uint32_t kv_it = 0;
+            uint32_t n_q[2] = {0, 0};     // uses of each Q buffer so far
+            for (int w = blockIdx.x; w < prm.n_work; w += gridDim.x) {
+                const int qpair = prm.n_qpairs - 1 - w / prm.BH;
+                const int bh = w % prm.BH;
+                const int q0 = qpair * 256;
+                const int T0 = n_tiles(q0), T1 = n_tiles(q0 + 128);
+                const int T = max(T0, T1);
+                for (int i = 0; i < 2; ++i) {
+                    if ((i == 0 ? T0 : T1) == 0) continue;
+                    if (n_q[i] > 0 && !pf_wait(&q_empty[i], (n_q[i] - 1) & 1, kWaitQEmpty, abort_flag)) goto done;
+                    ++n_q[i];
+                    mbar_arrive_expect_tx(&q_full[i], C::kTileBytes);
+                    for (int p = 0; p < C::kPanels; ++p)
+                        tma_load_3d(sQ + i * C::kTileBytes + p * C::kPanelBytes, &map_q, p * 64, q0 + i * 128, bh,
+                                    &q_full[i]);
+                }
+                for (int t = 0; t < T; ++t) {
+                    for (int kv = 0; kv < 2; ++kv, ++kv_it) {
+                        const int stage = kv_it % C::kStages;
+                        const uint32_t round = kv_it / C::kStages;
+                        if (round > 0 && !pf_wait(&kv_empty[stage], (round - 1) & 1, kWaitKVEmpty, abort_flag)) goto done;
+                        mbar_arrive_expect_tx(&kv_full[stage], C::kTileBytes);
+                        for (int p = 0; p < C::kPanels; ++p)
+                            tma_load_3d(sKV + stage * C::kTileBytes + p * C::kPanelBytes, kv == 0 ? &map_k : &map_v,
+                                        p * 64, t * 128, bh, &kv_full[stage]);
+                    }
+                }
+            }
+        }
+    } else if (warp == 12) {
+        // ================================================================ MMA issue
+        reg_dec<48>();
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = make_idesc(128, 128, 0);
+            constexpr uint32_t idesc_o = make_idesc(128, D, 1);
+            const uint32_t tS[2] = {tmem_base + C::kColS0, tmem_base + C::kColS1};
+            const uint32_t tO[2] = {tmem_base + C::kColO0, tmem_base + C::kColO1};
+            uint32_t kv_it = 0;
+            uint32_t n_p[2] = {0, 0}, n_or[2] = {0, 0}, n_qf[2] = {0, 0};
+            auto issue_S = [&](int i, int stage) {
+                const uint32_t qa = smem_u32(sQ + i * C::kTileBytes);
+                const uint32_t ka = smem_u32(sKV + stage * C::kTileBytes);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t off = (ks >> 2) * C::kPanelBytes + (ks & 3) * 32;
+                    mma_ss(tS[i], smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(ka + off, 16, 1024), idesc_s,
+                           ks > 0);
+                }
+            };
+            auto issue_PV = [&](int i, int stage, bool first) {
+                const uint32_t va = smem_u32(sKV + stage * C::kTileBytes);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    // 16 keys = two 8-key swizzle atoms of 1024 bytes; panels of 64 d-columns are
+                    // kPanelBytes apart (leading-dimension offset of the MN-major operand)
+                    mma_ts(tO[i], tS[i] + ks * 8, smem_desc_sw128(va + ks * 2048, C::kPanelBytes, 1024), idesc_o,
+                           (!first) || ks > 0);
+                }
+            };
+            for (int w = blockIdx.x; w < prm.n_work; w += gridDim.x) {
+                const int qpair = prm.n_qpairs - 1 - w / prm.BH;
+                const int q0 = qpair * 256;
+                const int Ti[2] = {n_tiles(q0), n_tiles(q0 + 128)};
+                const int T = max(Ti[0], Ti[1]);
+                // ring positions of this work item: K_t at kv_it + 2t, V_t at kv_it + 2t + 1
+                auto stage_of = [&](uint32_t it) { return (int)(it % C::kStages); };
+                auto parity_of = [&](uint32_t it) { return (it / C::kStages) & 1u; };
+                // S_i(0)
+                if (!pf_wait(&kv_full[stage_of(kv_it)], parity_of(kv_it), kWaitKVFull, abort_flag)) goto done;
+                for (int i = 0; i < 2; ++i) {
+                    if (Ti[i] == 0) continue;
+                    if (!pf_wait(&q_full[i], n_qf[i] & 1, kWaitQFull, abort_flag)) goto done;
+                    ++n_qf[i];
+                    tc_fence_after();
+                    issue_S(i, stage_of(kv_it));
+                    tc_commit(&s_full[i]);
+                    if (Ti[i] == 1) tc_commit(&q_empty[i]);
+                }
+                tc_commit(&kv_empty[stage_of(kv_it)]);
+                for (int t = 0; t < T; ++t) {
+                    const uint32_t it_v = kv_it + 2 * t + 1;
+                    const uint32_t it_kn = kv_it + 2 * t + 2;
+                    if (!pf_wait(&kv_full[stage_of(it_v)], parity_of(it_v), kWaitKVFull, abort_flag)) goto done;
+                    bool kn_ready = false;
+                    for (int i = 0; i < 2; ++i) {
+                        if (t < Ti[i]) {
+                            if (!pf_wait(&p_full[i], n_p[i] & 1, kWaitPFull, abort_flag)) goto done;
+                            ++n_p[i];
+                            if (!pf_wait(&o_ready[i], n_or[i] & 1, kWaitOReady, abort_flag)) goto done;
+                            ++n_or[i];
+                            tc_fence_after();
+                            issue_PV(i, stage_of(it_v), t == 0);
+                            tc_commit(&pv_done[i]);
+                        }
+                        if (t + 1 < Ti[i]) {
+                            if (!kn_ready) {
+                                if (!pf_wait(&kv_full[stage_of(it_kn)], parity_of(it_kn), kWaitKVFull, abort_flag)) goto done;
+                                kn_ready = true;
+                                tc_fence_after();
+                            }
+                            issue_S(i, stage_of(it_kn));
+                            tc_commit(&s_full[i]);
+                            if (t + 2 == Ti[i]) tc_commit(&q_empty[i]);
+                        }
+                    }
+                    tc_commit(&kv_empty[stage_of(it_v)]);
+                    if (t + 1 < T) tc_commit(&kv_empty[stage_of(it_kn)]);
+                }
+                kv_it += 2 * T;
+            }
+        }
+    } else if (warp < 8) {
+        // ================================================================ softmax (weight recurrence)
+        reg_inc<192>();
+        const int i = warp >> 2;                       // query tile of this warpgroup
+        const int row = threadIdx.x & 127;             // row within the tile = tensor-memory lane
+        const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem_base + (i == 0 ? C::kColS0 : C::kColS1) + lane_sel;
+        const float c = prm.scale_log2e;
+        uint32_t n_s = 0, n_ae = 0;
+        for (int w = blockIdx.x; w < prm.n_work; w += gridDim.x) {
+            const int qpair = prm.n_qpairs - 1 - w / prm.BH;
+            const int bh = w % prm.BH;
+            const int q0 = qpair * 256 + i * 128;
+            const int Ti = n_tiles(q0);
+            const int gi = q0 + row;                   // global query index of this thread's row
+            const int limit = prm.causal ? min(Nk, gi + 1) : Nk;   // keys [0, limit) are visible
+            float L = -INFINITY;                       // log2-domain state: L = (s_i - ln w_i) * log2(e)
+            for (int t = 0; t < Ti; ++t) {
+                if (!pf_wait(&s_full[i], n_s & 1, kWaitSFull, abort_flag)) goto done;
+                ++n_s;
+                tc_fence_after();
+                float s[128];
+#pragma unroll
+                for (int cb = 0; cb < 4; ++cb) tmem_ld32(tS + cb * 32, reinterpret_cast<uint32_t*>(s) + cb * 32);
+                tc_wait_ld();
+                const int n0 = t * 128;
+                if (n0 + 128 > Nk || (prm.causal && n0 + 127 > q0)) {
+#pragma unroll
+                    for (int j = 0; j < 128; ++j) s[j] = (n0 + j < limit) ? s[j] : (c >= 0.f ? -INFINITY : INFINITY);
+                }
+                // tile-local reference: max over {L_old, c*s_j}
+                float m0 = s[0], m1 = s[1], m2 = s[2], m3 = s[3];
+                if (c >= 0.f) {
+#pragma unroll
+                    for (int j = 4; j < 128; j += 4) {
+                        m0 = fmaxf(m0, s[j]); m1 = fmaxf(m1, s[j + 1]); m2 = fmaxf(m2, s[j + 2]); m3 = fmaxf(m3, s[j + 3]);
+                    }
+                    m0 = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+                } else {
+#pragma unroll
+                    for (int j = 4; j < 128; j += 4) {
+                        m0 = fminf(m0, s[j]); m1 = fminf(m1, s[j + 1]); m2 = fminf(m2, s[j + 2]); m3 = fminf(m3, s[j + 3]);
+                    }
+                    m0 = fminf(fminf(m0, m1), fminf(m2, m3));
+                }
+                const float ref = fmaxf(L, m0 * c);
+                const float nref = -ref;
+                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+                for (int j = 0; j < 128; j += 4) {
+                    s[j] = ex2(fmaf(s[j], c, nref));         a0 += s[j];
+                    s[j + 1] = ex2(fmaf(s[j + 1], c, nref)); a1 += s[j + 1];
+                    s[j + 2] = ex2(fmaf(s[j + 2], c, nref)); a2 += s[j + 2];
+                    s[j + 3] = ex2(fmaf(s[j + 3], c, nref)); a3 += s[j + 3];
+                }
+                const float e_old = ex2(L - ref);            // 0 for the first tile (L = -inf)
+                const float l = e_old + ((a0 + a1) + (a2 + a3));
+                const float inv = rcp(l);                    // the hidden division: one reciprocal per row and tile
+                L = ref + lg2(l);
+                if (t > 0) {
+                    // hand alpha = 1 - W = exp(L_old - L_new) to the correction warps
+                    if (n_ae > 0 && !pf_wait(&alpha_empty[i], (n_ae - 1) & 1, kWaitAlphaEmpty, abort_flag)) goto done;
+                    ++n_ae;
+                    sAlpha[i * 128 + row] = e_old * inv;
+                    mbar_arrive(&alpha_full[i]);
+                }
+                uint32_t pk[64];
+#pragma unroll
+                for (int j = 0; j < 64; ++j) pk[j] = pack_bf16x2(s[2 * j] * inv, s[2 * j + 1] * inv);
+                tmem_st32(tS, pk);
+                tmem_st32(tS + 32, pk + 32);
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(&p_full[i]);
+            }
+            if (prm.lse != nullptr && Ti > 0 && gi < Nq) prm.lse[(long long)bh * Nq + gi] = L * kLn2;
+        }
+    } else if (warp < 12) {
+        // ================================================================ correction + epilogue
+        reg_dec<80>();
+        const int row = threadIdx.x & 127;
+        const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tO[2] = {tmem_base + C::kColO0 + lane_sel, tmem_base + C::kColO1 + lane_sel};
+        uint32_t n_af[2] = {0, 0}, n_pv[2] = {0, 0};
+        for (int w = blockIdx.x; w < prm.n_work; w += gridDim.x) {
+            const int qpair = prm.n_qpairs - 1 - w / prm.BH;
+            const int bh = w % prm.BH;
+            const int q0 = qpair * 256;
+            const int Ti[2] = {n_tiles(q0), n_tiles(q0 + 128)};
+            const int T = max(Ti[0], Ti[1]);
+            // the O accumulators are free (the previous epilogue has read them)
+            for (int i = 0; i < 2; ++i)
+                if (Ti[i] > 0) { tc_fence_before(); mbar_arrive(&o_ready[i]); }
+            for (int t = 1; t < T; ++t) {
+                for (int i = 0; i < 2; ++i) {
+                    if (t >= Ti[i]) continue;
+                    if (!pf_wait(&alpha_full[i], n_af[i] & 1, kWaitAlphaFull, abort_flag)) goto done;
+                    ++n_af[i];
+                    const float alpha = sAlpha[i * 128 + row];
+                    mbar_arrive(&alpha_empty[i]);
+                    if (!pf_wait(&pv_done[i], n_pv[i] & 1, kWaitPVDone, abort_flag)) goto done;
+                    ++n_pv[i];
+                    tc_fence_after();
+                    // O <- alpha O   (the (1 - w) factor of Eq. out-final for the tile)
+#pragma unroll
+                    for (int cb = 0; cb < D / 32; ++cb) {
+                        float ov[32];
+                        tmem_ld32(tO[i] + cb * 32, reinterpret_cast<uint32_t*>(ov));
+                        tc_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) ov[j] *= alpha;
+                        tmem_st32(tO[i] + cb * 32, reinterpret_cast<const uint32_t*>(ov));
+                    }
+                    tc_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(&o_ready[i]);
+                }
+            }
+            // epilogue: O is already normalised - convert and store, no division
+            for (int i = 0; i < 2; ++i) {
+                if (Ti[i] == 0) continue;
+                if (!pf_wait(&pv_done[i], n_pv[i] & 1, kWaitPVDone, abort_flag)) goto done;
+                ++n_pv[i];
+                tc_fence_after();
+                const int gi = q0 + i * 128 + row;
+                const long long orow = ((long long)bh * Nq + gi) * D;
+#pragma unroll
+                for (int cb = 0; cb < D / 32; ++cb) {
+                    float ov[32];
+                    tmem_ld32(tO[i] + cb * 32, reinterpret_cast<uint32_t*>(ov));
+                    tc_wait_ld();
+                    if (gi < Nq) {
+                        if (prm.out_f32) {
+                            float4* dst = reinterpret_cast<float4*>(static_cast<float*>(prm.o) + orow + cb * 32);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) dst[j] = make_float4(ov[4 * j], ov[4 * j + 1], ov[4 * j + 2], ov[4 * j + 3]);
+                        } else {
+                            uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(prm.o) + orow + cb * 32);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                dst[j] = make_uint4(pack_bf16x2(ov[8 * j], ov[8 * j + 1]), pack_bf16x2(ov[8 * j + 2], ov[8 * j + 3]),
+                                                    pack_bf16x2(ov[8 * j + 4], ov[8 * j + 5]), pack_bf16x2(ov[8 * j + 6], ov[8 * j + 7]));
+                        }
+                    }
+                }
+            }
+        }
+    } else {
+        reg_dec<48>();
+    }
+
+done:
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, C::kTmemCols);
+    }
+}
+
+}  // namespace flashd

@@ -26,6 +26,16 @@ def pytest_collection_modifyitems(config, items):
             item.add_marker(skip)
 
 
+@pytest.fixture(scope="session")
+def flashd_lib():
+    """Build (if stale) and load the C-ABI CUDA library."""
+    from paper_2505_14201_b200 import build as _build
+    _build.build()
+    import paper_2505_14201_b200 as pkg
+    pkg.lib()
+    return pkg
+
+
 def read_golden(name):
     """Parse a ``key: v v v`` text fixture into {key: [Fraction, ...]}."""
     from fractions import Fraction
