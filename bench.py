@@ -1,0 +1,445 @@
+#!/usr/bin/env python
+"""Benchmark of the FLASH-D attention forward on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1|c2|c3|c4]
+                    [--impl ours|reference] [--no-extra]
+
+One step = one forward pass over one batch of the workload (default: the
+encoder-shaped bf16 configuration, B=8 H=12 N=1024 d=64).  Prints one JSON line.
+The attention path does not shard: with N > 1 every rank runs an independent
+replica on its own GPU and the value is the sum over replicas divided by the
+slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+L2_BYTES = 126e6
+NOMINAL_BF16_TFLOPS = 2250.0
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def f32(x: float) -> float:
+    return float(np.float32(x))
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["source"] = "fallback"
+    return p
+
+
+# ----------------------------------------------------------------------------- distributed helpers
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def reduce_max(value: float, world: int, device=None) -> float:
+    """Max over ranks of a per-rank scalar (identity when not distributed)."""
+    if world <= 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(units_per_rank: float, world: int, max_ms: float) -> float:
+    """Whole-job throughput: the units all ranks processed divided by the slowest rank's time."""
+    return units_per_rank * world / (max_ms * 1e-3)
+
+
+# ----------------------------------------------------------------------------- clocks sampler
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            busy = [x for x in sm if x >= 0.5 * max(sm)] or sm
+            out.update(sm_mhz=statistics.median(busy), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ----------------------------------------------------------------------------- oracle leg (CPU)
+def oracle_sample(w, target_s=12.0):
+    """Time the fp64 oracle, as it stands, on a bounded sample of workload ``w``:
+    the leading heads of the batch, every query row, every key.  Returns
+    (metric value in TFLOP/s, seconds, description, threads)."""
+    import torch
+    import oracle
+    from paper_2505_14201_b200 import synth
+    threads = oracle.num_threads()
+    # small probe to size the sample
+    probe = synth.Workload("probe", 1, 1, min(w.Nq, 256), min(w.Nk, 2048), w.d, w.causal, w.dtype, 99)
+    q, k, v = synth.make_inputs(probe)
+    t0 = time.perf_counter()
+    oracle.attn_naive(q, k, v, f32(w.scale), probe.causal)
+    dt = max(time.perf_counter() - t0, 1e-4)
+    rate = probe.flops / dt                               # counted flop/s of the oracle
+    per_head = w.flops / (w.B * w.H)
+    if per_head <= rate * target_s:
+        heads = max(1, min(w.B * w.H, int(rate * target_s / per_head)))
+        rows = w.Nq
+    else:
+        heads = 1
+        rows = max(1, int(w.Nq * rate * target_s / per_head))
+    g = torch.Generator().manual_seed(w.seed)
+    q = (torch.randn(1, heads, w.Nq, w.d, generator=g) * w.q_gain)
+    k = (torch.randn(1, heads, w.Nk, w.d, generator=g) * w.k_gain)
+    v = torch.randn(1, heads, w.Nk, w.d, generator=g)
+    if w.outlier_every:
+        k[:, :, :: w.outlier_every] *= w.outlier_gain
+    dt_ = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    q, k, v = q.to(dt_), k.to(dt_), v.to(dt_)
+    row_idx = list(range(w.Nq - rows, w.Nq))              # the last rows: the longest ones when causal
+    t0 = time.perf_counter()
+    oracle.attn_naive(q[:, :, row_idx], k, v, f32(w.scale), w.causal, q_index=row_idx)
+    secs = time.perf_counter() - t0
+    if w.causal:
+        pairs = sum(min(i + 1, w.Nk) for i in row_idx) * heads
+    else:
+        pairs = rows * w.Nk * heads
+    flops = 4.0 * pairs * w.d
+    desc = (f"oracle.attn_naive (fp64, OpenMP) on {heads} of {w.B * w.H} heads, last {rows} of {w.Nq} query rows, "
+            f"all {w.Nk} keys, same recipe as the workload; {secs:.1f} s")
+    return flops / secs / 1e12, secs, desc, threads
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle timed on the host cores (rank 0 only)."""
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    from paper_2505_14201_b200 import synth
+    w = synth.WORKLOADS[args.workload]
+    vals, secs_all, desc, threads = [], [], "", 1
+    budget = 150.0
+    per_step = min(12.0, budget / max(1, args.steps + args.warmup))
+    for i in range(args.warmup + args.steps):
+        val, secs, desc, threads = oracle_sample(w, target_s=per_step)
+        if i >= args.warmup:
+            vals.append(val); secs_all.append(secs)
+    value = statistics.mean(vals) if vals else 0.0
+    line = {
+        "impl": "reference", "metric": "attn_fwd_tflops", "value": value, "unit": "TFLOP/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * statistics.mean(secs_all) if secs_all else None,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, extra={"note": "each step is a bounded sample of the workload"}),
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w, extra=None):
+    c = {"workload": w.name, "B": w.B, "H": w.H, "Nq": w.Nq, "Nk": w.Nk, "d": w.d, "causal": w.causal,
+         "in_dtype": w.dtype, "scale": "1/sqrt(d)", "seed": w.seed}
+    if extra:
+        c.update(extra)
+    return c
+
+
+# ----------------------------------------------------------------------------- GPU legs
+def time_gpu(fn, steps, warmup, torch):
+    for i in range(warmup):
+        fn(i)
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        fn(warmup + i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1)
+
+
+def make_sets(w, device, min_bytes):
+    """Enough distinct input sets that one pass over all of them exceeds L2."""
+    import torch
+    from paper_2505_14201_b200 import synth
+    q, k, v = synth.make_inputs(w, device=device)
+    esz = q.element_size()
+    set_bytes = (2 * q.numel() + 2 * k.numel()) * esz
+    n = max(1, math.ceil(min_bytes / set_bytes))
+    sets = [(q, k, v, torch.empty_like(q))]
+    for i in range(1, n):
+        g = torch.Generator(device=device).manual_seed(1000 + w.seed * 16 + i)
+        perm = torch.randperm(w.Nk, device=device, generator=g)
+        sets.append((q.roll(i, dims=2).contiguous(), k[:, :, perm].contiguous(), v[:, :, perm].contiguous(),
+                     torch.empty_like(q)))
+    return sets, set_bytes
+
+
+def bench_workload(fd, w, steps, warmup, torch, device):
+    """Device-resident timing of one workload; returns a dict of results."""
+    sc = f32(w.scale)
+    if w.splitk:
+        q, k, v = make_c4(w, device)
+        S = fd.flashd_splitk_num_splits(w.B, w.H, w.Nq, w.Nk, w.d)
+        ws = torch.empty((w.B, w.H, w.Nq, S, w.d + 1), dtype=torch.float32, device=device)
+        o = torch.empty_like(q)
+        fn = lambda i: fd.flashd_attn_fwd_splitk(q, k, v, sc, S, workspace=ws, o=o)
+        n0 = fd.launch_count()
+        ms = time_gpu(fn, steps, warmup, torch)
+        launches = (fd.launch_count() - n0) * steps // (steps + warmup)
+        alg_bytes = w.kv_bytes
+        return {"ms_per_step": ms / steps, "tflops": w.flops * steps / (ms * 1e-3) / 1e12,
+                "gbs": alg_bytes * steps / (ms * 1e-3) / 1e9, "launches": launches, "num_splits": S,
+                "l2": "inputs (34 GB) exceed L2", "tensors": (q, k, v, o)}
+    sets, set_bytes = make_sets(w, device, 1.5 * L2_BYTES)
+    fn = lambda i: fd.flashd_attn_fwd(*sets[i % len(sets)][:3], sc, w.causal, o=sets[i % len(sets)][3])
+    n0 = fd.launch_count()
+    ms = time_gpu(fn, steps, warmup, torch)
+    launches = (fd.launch_count() - n0) * steps // (steps + warmup)
+    return {"ms_per_step": ms / steps, "tflops": w.flops * steps / (ms * 1e-3) / 1e12, "launches": launches,
+            "l2": f"rotating {len(sets)} input sets of {set_bytes / 1e6:.0f} MB (> 126 MB L2 in total)",
+            "tensors": sets[0]}
+
+
+def make_c4(w, device):
+    from paper_2505_14201_b200 import synth
+    return synth.make_inputs(w, device=device)
+
+
+def bench_e2e(fd, w, steps, warmup, torch):
+    """Same metric through the host-buffer C-ABI call: pinned host inputs, H2D,
+    kernel(s), D2H of the result, all inside the timed region."""
+    from paper_2505_14201_b200 import synth
+    if w.splitk:
+        # 34 GB of pinned host memory is not a sane benchmark input; time a
+        # batch slice (B = 4) and scale the metric by the work it covers
+        w = synth.Workload(w.name + " (B=4 slice)", 4, w.H, w.Nq, w.Nk, w.d, w.causal, w.dtype, w.seed,
+                           splitk=True, per_batch=True)
+    q, k, v = synth.make_inputs(w)
+    q, k, v = q.pin_memory(), k.pin_memory(), v.pin_memory()
+    o = torch.empty_like(q).pin_memory()
+    sc = f32(w.scale)
+    path = 2 if w.splitk else 0
+    t_steps = max(3, min(steps, 20))
+    for _ in range(max(3, min(warmup, 5))):
+        fd.flashd_attn_fwd_host(q, k, v, sc, w.causal, path=path, o=o)
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(t_steps):
+        fd.flashd_attn_fwd_host(q, k, v, sc, w.causal, path=path, o=o)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / t_steps
+    h2d = (q.numel() + k.numel() + v.numel()) * q.element_size()
+    d2h = o.numel() * o.element_size()
+    return {"tflops": w.flops / (ms * 1e-3) / 1e12, "ms_per_step": ms, "h2d": h2d, "d2h": d2h, "steps": t_steps,
+            "workload": w.name}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="c1", choices=["c1", "c2", "c3", "c4"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extra", action="store_true", help="skip the other configurations and the CPU baseline")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import paper_2505_14201_b200 as fd
+    from paper_2505_14201_b200 import synth
+
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=device)
+    fd.lib()
+    peaks = load_peaks()
+    w = synth.WORKLOADS[args.workload]
+
+    sampler = ClockSampler(local_rank)
+    # ---- headline: device-resident inputs
+    # build inputs, then barrier + sync, time K steps, sync + barrier, max over ranks
+    sc = f32(w.scale)
+    if w.splitk:
+        q, k, v = make_c4(w, device)
+        S = fd.flashd_splitk_num_splits(w.B, w.H, w.Nq, w.Nk, w.d)
+        ws = torch.empty((w.B, w.H, w.Nq, S, w.d + 1), dtype=torch.float32, device=device)
+        o = torch.empty_like(q)
+        step = lambda i: fd.flashd_attn_fwd_splitk(q, k, v, sc, S, workspace=ws, o=o)
+        l2_note = "inputs (34 GB) exceed L2"
+    else:
+        sets, set_bytes = make_sets(w, device, 1.5 * L2_BYTES)
+        step = lambda i: fd.flashd_attn_fwd(*sets[i % len(sets)][:3], sc, w.causal, o=sets[i % len(sets)][3])
+        l2_note = f"rotating {len(sets)} input sets of {set_bytes / 1e6:.0f} MB each (> 126 MB L2 in total)"
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler.start()
+    n0 = fd.launch_count()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    e1.record()
+    torch.cuda.synchronize()
+    launches = fd.launch_count() - n0
+    if world > 1:
+        dist.barrier()
+    local_ms = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    st, detail = fd.flashd_last_device_status()
+    if st != 0:
+        raise SystemExit(f"device status {st} {detail}")
+    max_ms = reduce_max(local_ms, world, device)
+    value = aggregate_value(w.flops * args.steps, world, max_ms) / 1e12
+    ms_per_step = max_ms / args.steps
+
+    # ---- roofline of the dominant kernel (one launch per step for prefill; partial kernel for decode)
+    if w.splitk:
+        alg = w.kv_bytes
+        achieved = alg / (local_ms / args.steps * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                "frac_of_nominal": achieved / NOMINAL_HBM_GBS,
+                "kernel": "splitk_partial_kernel (+combine, timed together)"}
+    else:
+        achieved = w.flops / (local_ms / args.steps * 1e-3) / 1e12
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["bf16_tflops"], "traffic": None, "peak_source": peaks["source"],
+                "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS, "kernel": f"prefill_kernel<{w.d}>"}
+
+    line = {
+        "metric": "attn_fwd_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": workload_config(w, {"l2": l2_note, "parallelism": "replicas only" if world > 1 else "1 gpu"}),
+        "roofline": roof, "clocks": clocks, "gpu_launches": int(launches),
+    }
+
+    if rank == 0:
+        e2e = bench_e2e(fd, w, args.steps, args.warmup, torch)
+        line["e2e"] = {"value": e2e["tflops"] * world, "unit": "TFLOP/s", "h2d_bytes_per_step": e2e["h2d"],
+                       "d2h_bytes_per_step": e2e["d2h"], "ms_per_step": e2e["ms_per_step"], "workload": e2e["workload"],
+                       "note": "flashd_attn_fwd_host: pinned host q,k,v -> device, kernel, o -> host, every step"}
+    if world > 1:
+        # replicas: every rank does the same end-to-end work; report rank 0's rate times the replica count
+        dist.barrier()
+
+    if rank == 0 and world == 1 and not args.no_extra:
+        # free the headline inputs before the larger configurations
+        others = {}
+        try:
+            del step
+            if w.splitk:
+                del q, k, v, ws, o
+            else:
+                del sets
+            torch.cuda.empty_cache()
+            for name in ("c1", "c2", "c3", "c4"):
+                if name == args.workload:
+                    continue
+                ow = synth.WORKLOADS[name]
+                free, _ = torch.cuda.mem_get_info()
+                if ow.splitk and free < 50e9:
+                    others[name] = {"skipped": "not enough free device memory"}
+                    continue
+                r = bench_workload(fd, ow, 5 if name in ("c3", "c4") else 20, 3, torch, device)
+                r.pop("tensors", None)
+                if ow.splitk:
+                    r["frac_hbm_measured"] = r["gbs"] / peaks["hbm_gbs"]
+                    r["frac_hbm_nominal"] = r["gbs"] / NOMINAL_HBM_GBS
+                else:
+                    r["frac_tensor_measured"] = r["tflops"] / peaks["bf16_tflops"]
+                    r["frac_tensor_nominal"] = r["tflops"] / NOMINAL_BF16_TFLOPS
+                others[name] = r
+                torch.cuda.empty_cache()
+        except Exception as ex:  # the headline number stands on its own
+            others["error"] = repr(ex)
+        line["other_configs"] = others
+        val, secs, desc, threads = oracle_sample(w, target_s=12.0)
+        line["cpu_baseline"] = {"value": val, "unit": "TFLOP/s", "cores": threads, "kind": "oracle", "sample": desc}
+
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
