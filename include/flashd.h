@@ -137,6 +137,44 @@ int flashd_attn_fwd_splitk(const void* q, const void* k, const void* v, void* o,
                            int num_splits, void* stream);
 
 /* ------------------------------------------------------------------------
+ * Split-K forward that allocates nothing.  (The paper has no counterpart: this
+ * entry point exists for integration reasons only.)
+ *
+ * Who needs it: a decode loop inside an inference server usually hands every
+ * byte of device memory to its own pool at start-up and runs each token under
+ * a fixed memory plan.  Such a caller has nowhere to take the split-K
+ * workspace from, and cudaMalloc inside the per-token call would either fail
+ * or stall the device while the driver maps memory.  Plugin hosts that forbid
+ * allocation inside the hot call are in the same position.
+ *
+ * Same computation and same kernels as flashd_attn_fwd_splitk, but the
+ * partial states live in a fixed array that is part of the library image
+ * (FLASHD_STATIC_SCRATCH_BYTES of device memory on every GPU that loads the
+ * library, held until the process exits).  The caller passes only inputs and
+ * the output.  The call makes no cudaMalloc / cudaFree and uses no allocating
+ * library routine.
+ *
+ * Limit: B*H*Nq*num_splits*(d+1)*4 bytes must not exceed
+ * FLASHD_STATIC_SCRATCH_BYTES; a larger problem is rejected with
+ * FLASHD_ERR_WORKSPACE and nothing is launched (num_splits <= 0 takes the
+ * library's choice first, then the check is made).
+ *
+ * First call on a device: it looks up the device address of the array (once
+ * per device, with that device current) before launching.  Make that first
+ * call before starting any stream capture.
+ *
+ * Sharing: every call on a device uses the same array, and the array keeps
+ * whatever the previous call left in it.  Nothing in it needs clearing - the
+ * partial kernel rewrites every (row, split) slot it later reads, empty splits
+ * included - but two calls whose kernels overlap on the GPU (different
+ * streams, or different host threads) race on it and give wrong results.
+ * Serialise such calls on one stream.                                      */
+#define FLASHD_STATIC_SCRATCH_BYTES (8u << 20)
+int flashd_attn_fwd_splitk_static(const void* q, const void* k, const void* v, void* o,
+                                  int B, int H, int Nq, int Nk, int d, float scale,
+                                  int num_splits, void* stream);
+
+/* ------------------------------------------------------------------------
  * End-to-end call on HOST buffers: q, k, v, o are host pointers (pinned
  * memory gives asynchronous copies).  The call allocates device buffers from
  * the stream-ordered pool of the current device, copies q, k, v in, runs the

@@ -17,8 +17,8 @@ MAX_SPLITS = 64
 EXPORTED_SYMBOLS = (
     "flashd_attn_fwd", "flashd_attn_fwd_ex", "flashd_attn_fwd_f32", "flashd_attn_fwd_perkey",
     "flashd_splitk_workspace_bytes", "flashd_splitk_num_splits", "flashd_splitk_partial",
-    "flashd_splitk_combine", "flashd_attn_fwd_splitk", "flashd_attn_fwd_host",
-    "flashd_last_device_status", "flashd_status_string", "flashd_version", "flashd_launch_count",
+    "flashd_splitk_combine", "flashd_attn_fwd_splitk", "flashd_attn_fwd_splitk_static",
+    "flashd_attn_fwd_host", "flashd_last_device_status", "flashd_status_string", "flashd_version", "flashd_launch_count",
 )
 
 _lock = threading.Lock()
@@ -59,6 +59,7 @@ def lib() -> ctypes.CDLL:
             L.flashd_splitk_partial.argtypes = [vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_splitk_combine.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, vp]
             L.flashd_attn_fwd_splitk.argtypes = [vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
+            L.flashd_attn_fwd_splitk_static.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_attn_fwd_host.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
             L.flashd_status_string.argtypes = [ci]
@@ -217,6 +218,27 @@ def flashd_attn_fwd_splitk(q, k, v, scale, num_splits=0, workspace=None, o=None,
     _check(lib().flashd_attn_fwd_splitk(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(workspace),
                                         workspace.numel() * workspace.element_size(), B, H, Nq, Nk, d,
                                         float(scale), int(num_splits), _stream_ptr(stream)), "flashd_attn_fwd_splitk")
+    return o
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def flashd_attn_fwd_splitk_static(q, k, v, scale, num_splits=0, o=None, stream=None):
+    """Split-K forward for callers that must not allocate device memory inside
+    the call (a server's per-token decode step running under a fixed memory
+    plan): the partial states go to a fixed array inside the library instead of
+    a caller workspace.  Problems whose partial states exceed
+    ``STATIC_SCRATCH_BYTES`` raise ``FlashdError`` (status 5).  Calls share that
+    array, so they must not overlap on the GPU.  Pass ``o`` to keep this wrapper
+    from allocating the output."""
+    import torch
+    B, H, Nq, Nk, d = _dims(q, k, v)
+    if o is None:
+        o = torch.empty_like(q)
+    _check(lib().flashd_attn_fwd_splitk_static(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, H, Nq, Nk, d,
+                                               float(scale), int(num_splits), _stream_ptr(stream)),
+           "flashd_attn_fwd_splitk_static")
     return o
 
 

@@ -159,6 +159,28 @@ int launch_partial(const void* q, const void* k, const void* v, void* ws, long l
     return after_launch();
 }
 
+// Scratch of the allocation-free split-K entry point: partial states
+// [rows, splits, d+1] fp32.  Part of the library image, so every device that
+// loads the library holds it until exit.  In host code this name is only a
+// handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) float g_static_scratch[FLASHD_STATIC_SCRATCH_BYTES / sizeof(float)];
+
+// Device address of g_static_scratch on the current device, looked up once per
+// device; nullptr if the lookup failed.
+float* static_scratch_ptr() {
+    static std::mutex mu;
+    static float* cached[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached[dev] == nullptr) {
+        float* ptr = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_scratch) != cudaSuccess) return nullptr;
+        cached[dev] = ptr;
+    }
+    return cached[dev];
+}
+
 int check_splits(int Nk, int num_splits) {
     if (num_splits < 1 || num_splits > FLASHD_MAX_SPLITS || num_splits > Nk) return FLASHD_ERR_WORKSPACE;
     // every split but the last must be non-empty by construction; the last one is
@@ -291,6 +313,30 @@ int flashd_attn_fwd_splitk(const void* q, const void* k, const void* v, void* o,
     int st = flashd_splitk_partial(q, k, v, workspace, workspace_bytes, B, H, Nq, Nk, d, scale, num_splits, stream);
     if (st != FLASHD_OK) return st;
     return flashd_splitk_combine(workspace, o, nullptr, B, H, Nq, d, num_splits, FLASHD_BF16, stream);
+}
+
+int flashd_attn_fwd_splitk_static(const void* q, const void* k, const void* v, void* o, int B, int H, int Nq,
+                                  int Nk, int d, float scale, int num_splits, void* stream) {
+    const int st = check_common(q, k, v, o, B, H, Nq, Nk, d, scale);
+    if (st != FLASHD_OK) return st;
+    if (d != 128 && d != 64) return FLASHD_ERR_UNSUPPORTED;
+    if (num_splits <= 0) num_splits = flashd_splitk_num_splits(B, H, Nq, Nk, d);
+    const int cs = check_splits(Nk, num_splits);
+    if (cs != FLASHD_OK) return cs;
+    const long long rows = (long long)B * H * Nq;
+    if (rows > 0x7fffffffLL) return FLASHD_ERR_SHAPE;
+    const unsigned long long need = (unsigned long long)rows * num_splits * (unsigned long long)(d + 1) * sizeof(float);
+    if (need > FLASHD_STATIC_SCRATCH_BYTES) return FLASHD_ERR_WORKSPACE;   // beyond the fixed scratch
+    float* ws = static_scratch_ptr();
+    if (ws == nullptr) return FLASHD_ERR_CUDA;
+    cudaStream_t s = as_stream(stream);
+    const int ps = (d == 128) ? launch_partial<128>(q, k, v, ws, rows, Nq, Nk, scale, num_splits, s)
+                              : launch_partial<64>(q, k, v, ws, rows, Nq, Nk, scale, num_splits, s);
+    if (ps != FLASHD_OK) return ps;
+    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(o);
+    if (d == 128) splitk_combine_kernel<128, __nv_bfloat16><<<(unsigned)rows, 128, 0, s>>>(ws, out, nullptr, num_splits);
+    else splitk_combine_kernel<64, __nv_bfloat16><<<(unsigned)rows, 64, 0, s>>>(ws, out, nullptr, num_splits);
+    return after_launch();
 }
 
 int flashd_attn_fwd_host(const void* q, const void* k, const void* v, void* o, int path, int B, int H, int Nq,
