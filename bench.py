@@ -305,6 +305,9 @@ def main():
     ap.add_argument("--workload", default="c1", choices=["c1", "c2", "c3", "c4"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the other configurations and the CPU baseline")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="override the workload's batch size B (smaller case for profiler captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -328,6 +331,9 @@ def main():
     fd.lib()
     peaks = load_peaks()
     w = synth.WORKLOADS[args.workload]
+    if args.batch > 0:
+        import dataclasses
+        w = dataclasses.replace(w, B=args.batch, name=f"{w.name} (B={args.batch})")
 
     sampler = ClockSampler(local_rank)
     # ---- headline: device-resident inputs
@@ -392,7 +398,7 @@ def main():
         "roofline": roof, "clocks": clocks, "gpu_launches": int(launches),
     }
 
-    if rank == 0:
+    if rank == 0 and not args.no_e2e:
         e2e = bench_e2e(fd, w, args.steps, args.warmup, torch)
         line["e2e"] = {"value": e2e["tflops"] * world, "unit": "TFLOP/s", "h2d_bytes_per_step": e2e["h2d"],
                        "d2h_bytes_per_step": e2e["d2h"], "ms_per_step": e2e["ms_per_step"], "workload": e2e["workload"],
