@@ -1,25 +1,33 @@
 // Tiled FLASH-D forward on the 5th-generation tensor cores (sm_100a).
 //
 // One CTA owns a pair of 128-row query tiles of one head and walks the key
-// sequence in tiles of 128 keys.  Per query tile and key tile:
+// sequence in tiles of 128 keys.  The per-key step of Algorithm 3 with the
+// division written out is, for x = s_i - L_{i-1} and L = s - ln w the carried state,
+//     w_i = sigma(x) = e^x / (1 + e^x)             Eq. (w-last)
+//     o_i = (o_{i-1} + e^x v_i) / (1 + e^x)        Eq. (out-final)
+// Applied to a tile of keys as one group this becomes, per query row,
+//     O_t = (O_{t-1} + sum_j e^{x_j} v_j) / (1 + sum_j e^{x_j}),   x_j = s_j - L_{t-1}
+//     L_t = L_{t-1} + ln(1 + sum_j e^{x_j})
+// and that is what the kernel evaluates (log2 units, c = scale*log2(e)):
 //   S = Q K^T                      tcgen05.mma, operands in shared memory (TMA),
 //                                  accumulator in tensor memory
-//   per row (one thread per row), with c = scale*log2(e) and L in log2 units:
-//       ref   = max(L_old, max_j c*s_j)          tile-local reference, not carried
-//       pt_j  = 2^(c*s_j - ref),  l = 2^(L_old - ref) + sum_j pt_j
-//       L_new = ref + log2 l                      = log-sum-exp of {L_old, s_j}
-//       P_j   = pt_j / l = exp(s_j - L_new)       weights of the tile's keys
-//       alpha = 2^(L_old - ref) / l = exp(L_old - L_new) = 1 - sum_j P_j
-//   O <- alpha O + P V             rescale by the correction warps, then
-//                                  tcgen05.mma with P read from tensor memory
-// This is Algorithm 3 of the paper applied to the tile as one super-key of score
-// L_T = log-sum-exp(s_j): Eq. (w-last) gives W = sigma(L_T - L_old), and
-// multiplying Eq. (out-final) through gives alpha = 1 - W and P_j = W exp(s_j - L_T).
-// O is normalised after every tile, the only carried state per row is L
-// (= s_i - ln w_i), there is no running maximum and no final division: the single
-// reciprocal 1/l per row and tile is the division hidden in the sigmoid.
+//   per row (one thread per row):
+//       ref   = max(L_{t-1}, max_j c*s_j)          tile-local reference, not carried;
+//                                                  equals L_{t-1} unless a new key dominates
+//       e_old = 2^(L_{t-1} - ref)                  (= 1 in the common case)
+//       pt_j  = 2^(c*s_j - ref)                    (= e^{x_j} in the common case)
+//       l_t   = e_old + sum_j pt_j ,  L_t = ref + log2 l_t
+//   O~_t = beta_t O~_{t-1} + Pt V    beta_t = e_old / l_{t-1}: the division that closes
+//                                    step t-1 is applied, as a reciprocal-multiply by the
+//                                    correction warps, when step t opens; so the
+//                                    accumulator holds the normalised output O_{t-1} (times
+//                                    e_old) while the new keys are added, and the last
+//                                    reciprocal 1/l_T is applied in the epilogue.
+// There is no running maximum and no separate softmax denominator: the state per row
+// is L alone (l_t is L_t - ref_t in the linear domain), one reciprocal per row and
+// tile plays the part of the sigmoid's division.
 //
-// Warp roles (16 warps): 0-3 softmax of query tile 0, 4-7 softmax of query tile 1,
+// Warp roles (16 warps): 0-3 weights of query tile 0, 4-7 weights of query tile 1,
 // 8-11 correction + epilogue, 12 MMA issue, 13 TMA loads, 14-15 idle.
 // Tensor memory (512 columns): S0 | S1 | O0 | O1; P_i overlays the first 64
 // columns of S_i as packed bf16 pairs.
@@ -80,22 +88,26 @@ __device__ __forceinline__ void tc_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                  : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate) {
+// D[tmem] (+)= A[smem] * B[smem]; descriptors passed as (low word, shared high word)
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                       uint32_t idesc, uint32_t accumulate) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate) {
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi,
+                                       uint32_t idesc, uint32_t accumulate) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 // 32 consecutive 32-bit columns of this thread's tensor-memory lane
@@ -126,10 +138,16 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
 template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
-// Shared-memory matrix descriptor, 128-byte swizzle.  lbo / sbo in bytes.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) |
-           (1ull << 46) | (2ull << 61);
+// Shared-memory matrix descriptor, 128-byte swizzle, split in two 32-bit words.
+// Low word: start address >> 4 (bits 0-13) and leading-dimension byte offset >> 4
+// (bits 16-29).  High word: stride-dimension byte offset >> 4 (bits 0-13),
+// descriptor version 1 (bit 14), swizzle mode 2 = 128 bytes (bits 29-31).  Moving
+// the start address inside a tile only changes the low word.
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t saddr, uint32_t lbo) {
+    return ((saddr & 0x3FFFFu) >> 4) | ((lbo >> 4) << 16);
+}
+__host__ __device__ constexpr uint32_t smem_desc_hi(uint32_t sbo) {
+    return (sbo >> 4) | (1u << 14) | (2u << 29);
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, A K-major, B K-major (b_mn = 0) or MN-major (1).
 __host__ __device__ constexpr uint32_t make_idesc(int M, int N, int b_mn) {
@@ -231,7 +249,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
     if (warp == 13) {
         // ================================================================ TMA loader
-        reg_dec<48>();
+        reg_dec<64>();
         if (lane == 0) {
             uint32_t kv_it = 0;
             uint32_t n_q[2] = {0, 0};     // uses of each Q buffer so far
@@ -265,7 +283,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
     } else if (warp == 12) {
         // ================================================================ MMA issue
-        reg_dec<48>();
+        reg_dec<64>();
         if (lane == 0) {
             constexpr uint32_t idesc_s = make_idesc(128, 128, 0);
             constexpr uint32_t idesc_o = make_idesc(128, D, 1);
@@ -273,24 +291,28 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             const uint32_t tO[2] = {tmem_base + C::kColO0, tmem_base + C::kColO1};
             uint32_t kv_it = 0;
             uint32_t n_p[2] = {0, 0}, n_or[2] = {0, 0}, n_qf[2] = {0, 0};
+            // descriptor words: Q and K tiles are K-major (8-row groups 1024 bytes apart),
+            // V tiles are MN-major (8-key groups 1024 bytes apart, 64-column panels
+            // kPanelBytes apart)
+            constexpr uint32_t desc_hi = smem_desc_hi(1024);
+            const uint32_t q_lo[2] = {smem_desc_lo(smem_u32(sQ), 16), smem_desc_lo(smem_u32(sQ + C::kTileBytes), 16)};
+            const uint32_t k_lo0 = smem_desc_lo(smem_u32(sKV), 16);
+            const uint32_t v_lo0 = smem_desc_lo(smem_u32(sKV), C::kPanelBytes);
             auto issue_S = [&](int i, int stage) {
-                const uint32_t qa = smem_u32(sQ + i * C::kTileBytes);
-                const uint32_t ka = smem_u32(sKV + stage * C::kTileBytes);
+                const uint32_t qa = q_lo[i];
+                const uint32_t ka = k_lo0 + stage * (C::kTileBytes >> 4);
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (ks >> 2) * C::kPanelBytes + (ks & 3) * 32;
-                    mma_ss(tS[i], smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(ka + off, 16, 1024), idesc_s,
-                           ks > 0);
+                    const uint32_t off = ((ks >> 2) * C::kPanelBytes + (ks & 3) * 32) >> 4;
+                    mma_ss(tS[i], qa + off, ka + off, desc_hi, idesc_s, ks > 0);
                 }
             };
             auto issue_PV = [&](int i, int stage, bool first) {
-                const uint32_t va = smem_u32(sKV + stage * C::kTileBytes);
+                const uint32_t va = v_lo0 + stage * (C::kTileBytes >> 4);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    // 16 keys = two 8-key swizzle atoms of 1024 bytes; panels of 64 d-columns are
-                    // kPanelBytes apart (leading-dimension offset of the MN-major operand)
-                    mma_ts(tO[i], tS[i] + ks * 8, smem_desc_sw128(va + ks * 2048, C::kPanelBytes, 1024), idesc_o,
-                           (!first) || ks > 0);
+                    // 16 keys = two 8-key swizzle atoms of 1024 bytes
+                    mma_ts(tO[i], tS[i] + ks * 8, va + ks * (2048 >> 4), desc_hi, idesc_o, (!first) || ks > 0);
                 }
             };
             for (int w = blockIdx.x; w < prm.n_work; w += gridDim.x) {
@@ -347,7 +369,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
     } else if (warp < 8) {
         // ================================================================ softmax (weight recurrence)
-        reg_inc<192>();
+        reg_inc<176>();
         const int i = warp >> 2;                       // query tile of this warpgroup
         const int row = threadIdx.x & 127;             // row within the tile = tensor-memory lane
         const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
@@ -362,6 +384,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             const int gi = q0 + row;                   // global query index of this thread's row
             const int limit = prm.causal ? min(Nk, gi + 1) : Nk;   // keys [0, limit) are visible
             float L = -INFINITY;                       // log2-domain state: L = (s_i - ln w_i) * log2(e)
+            float inv_l = 1.f;                         // 1 / l of the previous tile
             for (int t = 0; t < Ti; ++t) {
                 if (!pf_wait(&s_full[i], n_s & 1, kWaitSFull, abort_flag)) goto done;
                 ++n_s;
@@ -375,7 +398,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll
                     for (int j = 0; j < 128; ++j) s[j] = (n0 + j < limit) ? s[j] : (c >= 0.f ? -INFINITY : INFINITY);
                 }
-                // tile-local reference: max over {L_old, c*s_j}
+                // tile-local reference: max over {L_{t-1}, c*s_j}
                 float m0 = s[0], m1 = s[1], m2 = s[2], m3 = s[3];
                 if (c >= 0.f) {
 #pragma unroll
@@ -391,40 +414,50 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     m0 = fminf(fminf(m0, m1), fminf(m2, m3));
                 }
                 const float ref = fmaxf(L, m0 * c);
+                const float e_old = ex2(L - ref);            // 0 for the first tile (L = -inf), else usually 1
+                if (t > 0) {
+                    // beta = e_old / l_{t-1}: closes step t-1 (its division) and opens step t
+                    if (n_ae > 0 && !pf_wait(&alpha_empty[i], (n_ae - 1) & 1, kWaitAlphaEmpty, abort_flag)) goto done;
+                    ++n_ae;
+                    sAlpha[i * 128 + row] = e_old * inv_l;
+                    mbar_arrive(&alpha_full[i]);
+                }
                 const float nref = -ref;
                 float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-                for (int j = 0; j < 128; j += 4) {
-                    s[j] = ex2(fmaf(s[j], c, nref));         a0 += s[j];
-                    s[j + 1] = ex2(fmaf(s[j + 1], c, nref)); a1 += s[j + 1];
-                    s[j + 2] = ex2(fmaf(s[j + 2], c, nref)); a2 += s[j + 2];
-                    s[j + 3] = ex2(fmaf(s[j + 3], c, nref)); a3 += s[j + 3];
-                }
-                const float e_old = ex2(L - ref);            // 0 for the first tile (L = -inf)
-                const float l = e_old + ((a0 + a1) + (a2 + a3));
-                const float inv = rcp(l);                    // the hidden division: one reciprocal per row and tile
-                L = ref + lg2(l);
-                if (t > 0) {
-                    // hand alpha = 1 - W = exp(L_old - L_new) to the correction warps
-                    if (n_ae > 0 && !pf_wait(&alpha_empty[i], (n_ae - 1) & 1, kWaitAlphaEmpty, abort_flag)) goto done;
-                    ++n_ae;
-                    sAlpha[i * 128 + row] = e_old * inv;
-                    mbar_arrive(&alpha_full[i]);
-                }
-                uint32_t pk[64];
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t pk[32];
 #pragma unroll
-                for (int j = 0; j < 64; ++j) pk[j] = pack_bf16x2(s[2 * j] * inv, s[2 * j + 1] * inv);
-                tmem_st32(tS, pk);
-                tmem_st32(tS + 32, pk + 32);
+                    for (int j = 0; j < 64; j += 4) {
+                        const float p0 = ex2(fmaf(s[64 * h + j], c, nref));
+                        const float p1 = ex2(fmaf(s[64 * h + j + 1], c, nref));
+                        const float p2 = ex2(fmaf(s[64 * h + j + 2], c, nref));
+                        const float p3 = ex2(fmaf(s[64 * h + j + 3], c, nref));
+                        a0 += p0; a1 += p1; a2 += p2; a3 += p3;
+                        pk[j / 2] = pack_bf16x2(p0, p1);
+                        pk[j / 2 + 1] = pack_bf16x2(p2, p3);
+                    }
+                    tmem_st32(tS + 32 * h, pk);
+                }
+                const float l = e_old + ((a0 + a1) + (a2 + a3));
+                inv_l = rcp(l);                              // the hidden division: one reciprocal per row and tile
+                L = ref + lg2(l);
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(&p_full[i]);
+            }
+            if (Ti > 0) {
+                // the reciprocal that closes the last step goes to the epilogue
+                if (n_ae > 0 && !pf_wait(&alpha_empty[i], (n_ae - 1) & 1, kWaitAlphaEmpty, abort_flag)) goto done;
+                ++n_ae;
+                sAlpha[i * 128 + row] = inv_l;
+                mbar_arrive(&alpha_full[i]);
             }
             if (prm.lse != nullptr && Ti > 0 && gi < Nq) prm.lse[(long long)bh * Nq + gi] = L * kLn2;
         }
     } else if (warp < 12) {
         // ================================================================ correction + epilogue
-        reg_dec<80>();
+        reg_dec<96>();
         const int row = threadIdx.x & 127;
         const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tO[2] = {tmem_base + C::kColO0 + lane_sel, tmem_base + C::kColO1 + lane_sel};
@@ -443,29 +476,35 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     if (t >= Ti[i]) continue;
                     if (!pf_wait(&alpha_full[i], n_af[i] & 1, kWaitAlphaFull, abort_flag)) goto done;
                     ++n_af[i];
-                    const float alpha = sAlpha[i * 128 + row];
+                    const float beta = sAlpha[i * 128 + row];
                     mbar_arrive(&alpha_empty[i]);
                     if (!pf_wait(&pv_done[i], n_pv[i] & 1, kWaitPVDone, abort_flag)) goto done;
                     ++n_pv[i];
                     tc_fence_after();
-                    // O <- alpha O   (the (1 - w) factor of Eq. out-final for the tile)
+                    // O~ <- beta O~
 #pragma unroll
-                    for (int cb = 0; cb < D / 32; ++cb) {
-                        float ov[32];
-                        tmem_ld32(tO[i] + cb * 32, reinterpret_cast<uint32_t*>(ov));
+                    for (int cb = 0; cb < D / 64; ++cb) {
+                        float ov[64];
+                        tmem_ld32(tO[i] + cb * 64, reinterpret_cast<uint32_t*>(ov));
+                        tmem_ld32(tO[i] + cb * 64 + 32, reinterpret_cast<uint32_t*>(ov) + 32);
                         tc_wait_ld();
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) ov[j] *= alpha;
-                        tmem_st32(tO[i] + cb * 32, reinterpret_cast<const uint32_t*>(ov));
+                        for (int j = 0; j < 64; ++j) ov[j] *= beta;
+                        tmem_st32(tO[i] + cb * 64, reinterpret_cast<const uint32_t*>(ov));
+                        tmem_st32(tO[i] + cb * 64 + 32, reinterpret_cast<const uint32_t*>(ov) + 32);
                     }
                     tc_wait_st();
                     tc_fence_before();
                     mbar_arrive(&o_ready[i]);
                 }
             }
-            // epilogue: O is already normalised - convert and store, no division
+            // epilogue: apply the reciprocal of the last step, convert and store
             for (int i = 0; i < 2; ++i) {
                 if (Ti[i] == 0) continue;
+                if (!pf_wait(&alpha_full[i], n_af[i] & 1, kWaitAlphaFull, abort_flag)) goto done;
+                ++n_af[i];
+                const float inv_l = sAlpha[i * 128 + row];
+                mbar_arrive(&alpha_empty[i]);
                 if (!pf_wait(&pv_done[i], n_pv[i] & 1, kWaitPVDone, abort_flag)) goto done;
                 ++n_pv[i];
                 tc_fence_after();
@@ -476,6 +515,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     float ov[32];
                     tmem_ld32(tO[i] + cb * 32, reinterpret_cast<uint32_t*>(ov));
                     tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) ov[j] *= inv_l;
                     if (gi < Nq) {
                         if (prm.out_f32) {
                             float4* dst = reinterpret_cast<float4*>(static_cast<float*>(prm.o) + orow + cb * 32);
@@ -493,7 +534,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             }
         }
     } else {
-        reg_dec<48>();
+        reg_dec<64>();
     }
 
 done:
