@@ -60,14 +60,17 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t by
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                  : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+// One wait attempt: the hardware may suspend the thread until the phase with the
+// given parity completes or about `hint_ns` nanoseconds have passed, so a waiting
+// warp does not take issue slots from the warps that share its scheduler.
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, uint32_t hint_ns = 20000u) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
         : "memory");
     return ok != 0;
 }
@@ -82,17 +85,13 @@ __device__ __forceinline__ uint64_t global_ns() {
 // seconds of wall time.  Returns false (after recording the failure) when the
 // wait ran out; the caller must then stop touching shared state and leave its
 // loop.
-constexpr uint32_t kSpinFast = 4096;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int which) {
-    for (uint32_t it = 0; it < kSpinFast; ++it)
-        if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_ns();
-    uint32_t it = 0;
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
-        __nanosleep(128);
-        if ((++it & 63u) == 0 && global_ns() - t0 > kWaitLimitNs) break;
+        if (global_ns() - t0 > kWaitLimitNs) break;
     }
     report_timeout(which, parity);
     return false;

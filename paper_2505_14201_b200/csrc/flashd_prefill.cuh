@@ -166,19 +166,16 @@ struct PrefillParams {
     int n_work;         // BH * n_qpairs
 };
 
-// Wait bounded by an iteration count; also leaves when another thread of the
-// CTA has raised the abort flag.
+// Wait bounded to about two seconds; also leaves when another thread of the CTA
+// has raised the abort flag.
 __device__ __forceinline__ bool pf_wait(uint64_t* bar, uint32_t parity, unsigned int which,
                                         volatile uint32_t* abort_flag) {
-    for (uint32_t it = 0; it < kSpinFast; ++it)
-        if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_ns();
-    uint32_t it = 0;
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        __nanosleep(64);
-        if ((++it & 63u) == 0 && global_ns() - t0 > kWaitLimitNs) break;
+        if (global_ns() - t0 > kWaitLimitNs) break;
     }
     report_timeout(which, parity);
     *abort_flag = 1;
