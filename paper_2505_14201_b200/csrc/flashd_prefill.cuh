@@ -110,6 +110,24 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_
         ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// Same with ready-made 64-bit descriptors: one instruction per product, nothing to compute at issue time
+__device__ __forceinline__ void mma_ss64(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                         uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void mma_ts64(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                         uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | lo; }
 // 32 consecutive 32-bit columns of this thread's tensor-memory lane
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
     asm volatile(
@@ -246,7 +264,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
     if (warp == 13) {
         // ================================================================ TMA loader
-        reg_dec<64>();
+        reg_dec<96>();
         if (lane == 0) {
             uint32_t kv_it = 0;
             uint32_t n_q[2] = {0, 0};     // uses of each Q buffer so far
@@ -280,7 +298,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
     } else if (warp == 12) {
         // ================================================================ MMA issue
-        reg_dec<64>();
+        reg_dec<96>();
         if (lane == 0) {
             constexpr uint32_t idesc_s = make_idesc(128, 128, 0);
             constexpr uint32_t idesc_o = make_idesc(128, D, 1);
@@ -295,22 +313,34 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             const uint32_t q_lo[2] = {smem_desc_lo(smem_u32(sQ), 16), smem_desc_lo(smem_u32(sQ + C::kTileBytes), 16)};
             const uint32_t k_lo0 = smem_desc_lo(smem_u32(sKV), 16);
             const uint32_t v_lo0 = smem_desc_lo(smem_u32(sKV), C::kPanelBytes);
-            auto issue_S = [&](int i, int stage) {
+            // The issuing thread shares its scheduler with busy warps, so every instruction it
+            // needs between two products delays the tensor pipe.  The descriptors of the next
+            // products are therefore built while the thread would wait anyway (prep_*), and the
+            // products themselves are issued back to back from registers (fire_*).
+            constexpr int KS = D / 16;
+            uint64_t qd[KS], kd[KS], vd[8];
+            auto prep_S = [&](int i, int stage) {
                 const uint32_t qa = q_lo[i];
                 const uint32_t ka = k_lo0 + stage * (C::kTileBytes >> 4);
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
+                for (int ks = 0; ks < KS; ++ks) {
                     const uint32_t off = ((ks >> 2) * C::kPanelBytes + (ks & 3) * 32) >> 4;
-                    mma_ss(tS[i], qa + off, ka + off, desc_hi, idesc_s, ks > 0);
+                    qd[ks] = desc64(qa + off, desc_hi);
+                    kd[ks] = desc64(ka + off, desc_hi);
                 }
             };
-            auto issue_PV = [&](int i, int stage, bool first) {
+            auto fire_S = [&](int i) {
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) mma_ss64(tS[i], qd[ks], kd[ks], idesc_s, ks > 0);
+            };
+            auto prep_PV = [&](int stage) {
                 const uint32_t va = v_lo0 + stage * (C::kTileBytes >> 4);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    // 16 keys = two 8-key swizzle atoms of 1024 bytes
-                    mma_ts(tO[i], tS[i] + ks * 8, va + ks * (2048 >> 4), desc_hi, idesc_o, (!first) || ks > 0);
-                }
+                for (int ks = 0; ks < 8; ++ks) vd[ks] = desc64(va + ks * (2048 >> 4), desc_hi);   // 16 keys = two 1024-byte atoms
+            };
+            auto fire_PV = [&](int i, bool first) {
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) mma_ts64(tO[i], tS[i] + ks * 8, vd[ks], idesc_o, (!first) || ks > 0);
             };
             for (int w = blockIdx.x; w < prm.n_work; w += gridDim.x) {
                 const int qpair = prm.n_qpairs - 1 - w / prm.BH;
@@ -327,7 +357,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     if (!pf_wait(&q_full[i], n_qf[i] & 1, kWaitQFull, abort_flag)) goto done;
                     ++n_qf[i];
                     tc_fence_after();
-                    issue_S(i, stage_of(kv_it));
+                    prep_S(i, stage_of(kv_it));
+                    fire_S(i);
                     tc_commit(&s_full[i]);
                     if (Ti[i] == 1) tc_commit(&q_empty[i]);
                 }
@@ -338,13 +369,15 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     if (!pf_wait(&kv_full[stage_of(it_v)], parity_of(it_v), kWaitKVFull, abort_flag)) goto done;
                     bool kn_ready = false;
                     for (int i = 0; i < 2; ++i) {
+                        if (t < Ti[i]) prep_PV(stage_of(it_v));
+                        if (t + 1 < Ti[i]) prep_S(i, stage_of(it_kn));
                         if (t < Ti[i]) {
                             if (!pf_wait(&p_full[i], n_p[i] & 1, kWaitPFull, abort_flag)) goto done;
                             ++n_p[i];
                             if (!pf_wait(&o_ready[i], n_or[i] & 1, kWaitOReady, abort_flag)) goto done;
                             ++n_or[i];
                             tc_fence_after();
-                            issue_PV(i, stage_of(it_v), t == 0);
+                            fire_PV(i, t == 0);
                             tc_commit(&pv_done[i]);
                         }
                         if (t + 1 < Ti[i]) {
@@ -353,7 +386,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                                 kn_ready = true;
                                 tc_fence_after();
                             }
-                            issue_S(i, stage_of(it_kn));
+                            fire_S(i);
                             tc_commit(&s_full[i]);
                             if (t + 2 == Ti[i]) tc_commit(&q_empty[i]);
                         }
@@ -366,7 +399,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
     } else if (warp < 8) {
         // ================================================================ softmax (weight recurrence)
-        reg_inc<176>();
+        reg_inc<168>();
         const int i = warp >> 2;                       // query tile of this warpgroup
         const int row = threadIdx.x & 127;             // row within the tile = tensor-memory lane
         const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
@@ -396,19 +429,15 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     for (int j = 0; j < 128; ++j) s[j] = (n0 + j < limit) ? s[j] : (c >= 0.f ? -INFINITY : INFINITY);
                 }
                 // tile-local reference: max over {L_{t-1}, c*s_j}
-                float m0 = s[0], m1 = s[1], m2 = s[2], m3 = s[3];
+                float m0 = s[0], m1 = s[1];
                 if (c >= 0.f) {
 #pragma unroll
-                    for (int j = 4; j < 128; j += 4) {
-                        m0 = fmaxf(m0, s[j]); m1 = fmaxf(m1, s[j + 1]); m2 = fmaxf(m2, s[j + 2]); m3 = fmaxf(m3, s[j + 3]);
-                    }
-                    m0 = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+                    for (int j = 2; j < 126; j += 4) { m0 = max3(m0, s[j], s[j + 1]); m1 = max3(m1, s[j + 2], s[j + 3]); }
+                    m0 = max3(m0, m1, fmaxf(s[126], s[127]));
                 } else {
 #pragma unroll
-                    for (int j = 4; j < 128; j += 4) {
-                        m0 = fminf(m0, s[j]); m1 = fminf(m1, s[j + 1]); m2 = fminf(m2, s[j + 2]); m3 = fminf(m3, s[j + 3]);
-                    }
-                    m0 = fminf(fminf(m0, m1), fminf(m2, m3));
+                    for (int j = 2; j < 126; j += 4) { m0 = min3(m0, s[j], s[j + 1]); m1 = min3(m1, s[j + 2], s[j + 3]); }
+                    m0 = min3(m0, m1, fminf(s[126], s[127]));
                 }
                 const float ref = fmaxf(L, m0 * c);
                 const float e_old = ex2(L - ref);            // 0 for the first tile (L = -inf), else usually 1
@@ -419,23 +448,27 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     sAlpha[i * 128 + row] = e_old * inv_l;
                     mbar_arrive(&alpha_full[i]);
                 }
-                const float nref = -ref;
-                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+                const uint64_t c2 = pack2(c, c), nref2 = pack2(-ref, -ref);
+                uint64_t acc0 = pack2(0.f, 0.f), acc1 = acc0;
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     uint32_t pk[32];
 #pragma unroll
                     for (int j = 0; j < 64; j += 4) {
-                        const float p0 = ex2(fmaf(s[64 * h + j], c, nref));
-                        const float p1 = ex2(fmaf(s[64 * h + j + 1], c, nref));
-                        const float p2 = ex2(fmaf(s[64 * h + j + 2], c, nref));
-                        const float p3 = ex2(fmaf(s[64 * h + j + 3], c, nref));
-                        a0 += p0; a1 += p1; a2 += p2; a3 += p3;
+                        float x0, x1, x2, x3;
+                        unpack2(fma2(pack2(s[64 * h + j], s[64 * h + j + 1]), c2, nref2), x0, x1);
+                        unpack2(fma2(pack2(s[64 * h + j + 2], s[64 * h + j + 3]), c2, nref2), x2, x3);
+                        const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+                        acc0 = add2(acc0, pack2(p0, p1));
+                        acc1 = add2(acc1, pack2(p2, p3));
                         pk[j / 2] = pack_bf16x2(p0, p1);
                         pk[j / 2 + 1] = pack_bf16x2(p2, p3);
                     }
                     tmem_st32(tS + 32 * h, pk);
                 }
+                float a0, a1, a2, a3;
+                unpack2(acc0, a0, a1);
+                unpack2(acc1, a2, a3);
                 const float l = e_old + ((a0 + a1) + (a2 + a3));
                 inv_l = rcp(l);                              // the hidden division: one reciprocal per row and tile
                 L = ref + lg2(l);
@@ -454,7 +487,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
     } else if (warp < 12) {
         // ================================================================ correction + epilogue
-        reg_dec<96>();
+        reg_dec<80>();
         const int row = threadIdx.x & 127;
         const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tO[2] = {tmem_base + C::kColO0 + lane_sel, tmem_base + C::kColO1 + lane_sel};
@@ -480,15 +513,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     tc_fence_after();
                     // O~ <- beta O~
 #pragma unroll
-                    for (int cb = 0; cb < D / 64; ++cb) {
-                        float ov[64];
-                        tmem_ld32(tO[i] + cb * 64, reinterpret_cast<uint32_t*>(ov));
-                        tmem_ld32(tO[i] + cb * 64 + 32, reinterpret_cast<uint32_t*>(ov) + 32);
+                    for (int cb = 0; cb < D / 32; ++cb) {
+                        float ov[32];
+                        tmem_ld32(tO[i] + cb * 32, reinterpret_cast<uint32_t*>(ov));
                         tc_wait_ld();
 #pragma unroll
-                        for (int j = 0; j < 64; ++j) ov[j] *= beta;
-                        tmem_st32(tO[i] + cb * 64, reinterpret_cast<const uint32_t*>(ov));
-                        tmem_st32(tO[i] + cb * 64 + 32, reinterpret_cast<const uint32_t*>(ov) + 32);
+                        for (int j = 0; j < 32; ++j) ov[j] *= beta;
+                        tmem_st32(tO[i] + cb * 32, reinterpret_cast<const uint32_t*>(ov));
                     }
                     tc_wait_st();
                     tc_fence_before();
@@ -531,7 +562,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             }
         }
     } else {
-        reg_dec<64>();
+        reg_dec<96>();
     }
 
 done:
