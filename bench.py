@@ -452,7 +452,12 @@ def main():
                 if ow.splitk and free < 50e9:
                     others[name] = {"skipped": "not enough free device memory"}
                     continue
-                r = bench_workload(fd, ow, 5 if name in ("c3", "c4") else 20, 3, torch, device)
+                smp = ClockSampler(local_rank)
+                smp.start()
+                smp.mark_start()
+                r = bench_workload(fd, ow, 30 if name in ("c3", "c4") else 200, 3, torch, device)
+                smp.mark_end()
+                r["clocks"] = smp.stop()
                 r.pop("tensors", None)
                 if ow.splitk:
                     r["frac_hbm_measured"] = r["gbs"] / peaks["hbm_gbs"]

@@ -51,14 +51,14 @@ struct PrefillCfg {
     static constexpr int kStages = (D == 128) ? 4 : 6;           // K/V ring
     static constexpr int kThreads = 512;
     static constexpr int kBarriers = 16 + 2 * kStages;
-    static constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + 2 * 128 * 4 + kBarriers * 8 + 64 + 1024;
+    static constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + 2 * 2 * 128 * 4 + kBarriers * 8 + 64 + 1024;
     static constexpr uint32_t kTmemCols = 512;
     static constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO0 = 256, kColO1 = 256 + D;
 };
 
 enum {
     kWaitQFull = 0x200, kWaitQEmpty, kWaitKVFull, kWaitKVEmpty, kWaitSFull, kWaitPFull,
-    kWaitAlphaFull, kWaitAlphaEmpty, kWaitPVDone, kWaitOReady
+    kWaitAlphaFull, kWaitPVDone, kWaitOReady
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -210,14 +210,17 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     unsigned char* sQ = smem;                               // 2 tiles
     unsigned char* sKV = smem + 2 * C::kTileBytes;          // kStages tiles
-    float* sAlpha = reinterpret_cast<float*>(sKV + C::kStages * C::kTileBytes);   // [2][128]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sAlpha + 256);
+    // Per-row factors handed from the weights warps to the correction warps, [slot][tile][row].
+    // Two slots used alternately: message n of a tile is written only after the product that
+    // needed message n-1 has been issued, and that product waits for the correction warps to
+    // have consumed message n-1, so message n-2 (same slot) is never overwritten unread.
+    float* sAlpha = reinterpret_cast<float*>(sKV + C::kStages * C::kTileBytes);   // [2][2][128]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sAlpha + 512);
     uint64_t* q_full = bars;            // [2]
     uint64_t* q_empty = bars + 2;       // [2]
     uint64_t* s_full = bars + 4;        // [2]
     uint64_t* p_full = bars + 6;        // [2]
     uint64_t* alpha_full = bars + 8;    // [2]
-    uint64_t* alpha_empty = bars + 10;  // [2]
     uint64_t* pv_done = bars + 12;      // [2]
     uint64_t* o_ready = bars + 14;      // [2]
     uint64_t* kv_full = bars + 16;                 // [kStages]
@@ -235,7 +238,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             mbar_init(&s_full[i], 1);
             mbar_init(&p_full[i], 128);
             mbar_init(&alpha_full[i], 128);
-            mbar_init(&alpha_empty[i], 128);
             mbar_init(&pv_done[i], 1);
             mbar_init(&o_ready[i], 128);
         }
@@ -443,9 +445,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 const float e_old = ex2(L - ref);            // 0 for the first tile (L = -inf), else usually 1
                 if (t > 0) {
                     // beta = e_old / l_{t-1}: closes step t-1 (its division) and opens step t
-                    if (n_ae > 0 && !pf_wait(&alpha_empty[i], (n_ae - 1) & 1, kWaitAlphaEmpty, abort_flag)) goto done;
+                    sAlpha[(n_ae & 1) * 256 + i * 128 + row] = e_old * inv_l;
                     ++n_ae;
-                    sAlpha[i * 128 + row] = e_old * inv_l;
                     mbar_arrive(&alpha_full[i]);
                 }
                 const uint64_t c2 = pack2(c, c), nref2 = pack2(-ref, -ref);
@@ -478,9 +479,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             }
             if (Ti > 0) {
                 // the reciprocal that closes the last step goes to the epilogue
-                if (n_ae > 0 && !pf_wait(&alpha_empty[i], (n_ae - 1) & 1, kWaitAlphaEmpty, abort_flag)) goto done;
+                sAlpha[(n_ae & 1) * 256 + i * 128 + row] = inv_l;
                 ++n_ae;
-                sAlpha[i * 128 + row] = inv_l;
                 mbar_arrive(&alpha_full[i]);
             }
             if (prm.lse != nullptr && Ti > 0 && gi < Nq) prm.lse[(long long)bh * Nq + gi] = L * kLn2;
@@ -505,9 +505,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 for (int i = 0; i < 2; ++i) {
                     if (t >= Ti[i]) continue;
                     if (!pf_wait(&alpha_full[i], n_af[i] & 1, kWaitAlphaFull, abort_flag)) goto done;
+                    const float beta = sAlpha[(n_af[i] & 1) * 256 + i * 128 + row];
                     ++n_af[i];
-                    const float beta = sAlpha[i * 128 + row];
-                    mbar_arrive(&alpha_empty[i]);
                     if (!pf_wait(&pv_done[i], n_pv[i] & 1, kWaitPVDone, abort_flag)) goto done;
                     ++n_pv[i];
                     tc_fence_after();
@@ -530,9 +529,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             for (int i = 0; i < 2; ++i) {
                 if (Ti[i] == 0) continue;
                 if (!pf_wait(&alpha_full[i], n_af[i] & 1, kWaitAlphaFull, abort_flag)) goto done;
+                const float inv_l = sAlpha[(n_af[i] & 1) * 256 + i * 128 + row];
                 ++n_af[i];
-                const float inv_l = sAlpha[i * 128 + row];
-                mbar_arrive(&alpha_empty[i]);
                 if (!pf_wait(&pv_done[i], n_pv[i] & 1, kWaitPVDone, abort_flag)) goto done;
                 ++n_pv[i];
                 tc_fence_after();
