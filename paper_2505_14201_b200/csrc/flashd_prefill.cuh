@@ -50,8 +50,8 @@ struct PrefillCfg {
     static constexpr int kTileBytes = kPanels * kPanelBytes;     // one Q / K / V tile
     static constexpr int kStages = (D == 128) ? 4 : 6;           // K/V ring
     static constexpr int kThreads = 512;
-    static constexpr int kBarriers = 16 + 2 * kStages;
-    static constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + 2 * 2 * 128 * 4 + kBarriers * 8 + 64 + 1024;
+    static constexpr int kBarriers = 18 + 2 * kStages;
+    static constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + 3 * 2 * 128 * 4 + kBarriers * 8 + 64 + 1024;
     static constexpr uint32_t kTmemCols = 512;
     static constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO0 = 256, kColO1 = 256 + D;
 };
@@ -214,8 +214,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // Two slots used alternately: message n of a tile is written only after the product that
     // needed message n-1 has been issued, and that product waits for the correction warps to
     // have consumed message n-1, so message n-2 (same slot) is never overwritten unread.
+    // The reciprocal that closes the last step of a work item travels on a channel of its own
+    // (sFinal / final_full): it is posted without waiting for anything, so on the shared channel
+    // it could complete a second barrier phase before the first one was observed.
     float* sAlpha = reinterpret_cast<float*>(sKV + C::kStages * C::kTileBytes);   // [2][2][128]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sAlpha + 512);
+    float* sFinal = sAlpha + 512;                                                  // [2][128]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sFinal + 256);
     uint64_t* q_full = bars;            // [2]
     uint64_t* q_empty = bars + 2;       // [2]
     uint64_t* s_full = bars + 4;        // [2]
@@ -223,8 +227,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     uint64_t* alpha_full = bars + 8;    // [2]
     uint64_t* pv_done = bars + 12;      // [2]
     uint64_t* o_ready = bars + 14;      // [2]
-    uint64_t* kv_full = bars + 16;                 // [kStages]
-    uint64_t* kv_empty = bars + 16 + C::kStages;   // [kStages]
+    uint64_t* final_full = bars + 16;   // [2]
+    uint64_t* kv_full = bars + 18;                 // [kStages]
+    uint64_t* kv_empty = bars + 18 + C::kStages;   // [kStages]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::kBarriers);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
@@ -238,6 +243,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             mbar_init(&s_full[i], 1);
             mbar_init(&p_full[i], 128);
             mbar_init(&alpha_full[i], 128);
+            mbar_init(&final_full[i], 128);
             mbar_init(&pv_done[i], 1);
             mbar_init(&o_ready[i], 128);
         }
@@ -479,9 +485,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             }
             if (Ti > 0) {
                 // the reciprocal that closes the last step goes to the epilogue
-                sAlpha[(n_ae & 1) * 256 + i * 128 + row] = inv_l;
-                ++n_ae;
-                mbar_arrive(&alpha_full[i]);
+                sFinal[i * 128 + row] = inv_l;
+                mbar_arrive(&final_full[i]);
             }
             if (prm.lse != nullptr && Ti > 0 && gi < Nq) prm.lse[(long long)bh * Nq + gi] = L * kLn2;
         }
@@ -491,7 +496,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const int row = threadIdx.x & 127;
         const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tO[2] = {tmem_base + C::kColO0 + lane_sel, tmem_base + C::kColO1 + lane_sel};
-        uint32_t n_af[2] = {0, 0}, n_pv[2] = {0, 0};
+        uint32_t n_af[2] = {0, 0}, n_pv[2] = {0, 0}, n_fin[2] = {0, 0};
         for (int w = blockIdx.x; w < prm.n_work; w += gridDim.x) {
             const int qpair = prm.n_qpairs - 1 - w / prm.BH;
             const int bh = w % prm.BH;
@@ -528,9 +533,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             // epilogue: apply the reciprocal of the last step, convert and store
             for (int i = 0; i < 2; ++i) {
                 if (Ti[i] == 0) continue;
-                if (!pf_wait(&alpha_full[i], n_af[i] & 1, kWaitAlphaFull, abort_flag)) goto done;
-                const float inv_l = sAlpha[(n_af[i] & 1) * 256 + i * 128 + row];
-                ++n_af[i];
+                if (!pf_wait(&final_full[i], n_fin[i] & 1, kWaitAlphaFull, abort_flag)) goto done;
+                const float inv_l = sFinal[i * 128 + row];
+                ++n_fin[i];
                 if (!pf_wait(&pv_done[i], n_pv[i] & 1, kWaitPVDone, abort_flag)) goto done;
                 ++n_pv[i];
                 tc_fence_after();
