@@ -50,15 +50,21 @@ struct PrefillCfg {
     static constexpr int kTileBytes = kPanels * kPanelBytes;     // one Q / K / V tile
     static constexpr int kStages = (D == 128) ? 4 : 6;           // K/V ring
     static constexpr int kThreads = 512;
-    static constexpr int kBarriers = 18 + 2 * kStages;
+    static constexpr int kBarriers = 20 + 2 * kStages;
     static constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + 3 * 2 * 128 * 4 + kBarriers * 8 + 64 + 1024;
     static constexpr uint32_t kTmemCols = 512;
-    static constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO0 = 256, kColO1 = 256 + D;
+    // At D = 64 tensor memory has room for P next to S (S0 S1 P0 P1 O0 O1 = 512 columns), so
+    // the score product of step t+1 can run while the weights of step t are computed
+    // (lookahead 2).  At D = 128 P has to overlay S and S(t+1) follows P V(t) (lookahead 1).
+    static constexpr int kLookahead = (D == 64) ? 2 : 1;
+    static constexpr uint32_t kColS0 = 0, kColS1 = 128;
+    static constexpr uint32_t kColP0 = (D == 64) ? 256 : kColS0, kColP1 = (D == 64) ? 320 : kColS1;
+    static constexpr uint32_t kColO0 = (D == 64) ? 384 : 256, kColO1 = kColO0 + D;
 };
 
 enum {
     kWaitQFull = 0x200, kWaitQEmpty, kWaitKVFull, kWaitKVEmpty, kWaitSFull, kWaitPFull,
-    kWaitAlphaFull, kWaitPVDone, kWaitOReady
+    kWaitAlphaFull, kWaitPVDone, kWaitOReady, kWaitSFree
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -228,8 +234,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     uint64_t* pv_done = bars + 12;      // [2]
     uint64_t* o_ready = bars + 14;      // [2]
     uint64_t* final_full = bars + 16;   // [2]
-    uint64_t* kv_full = bars + 18;                 // [kStages]
-    uint64_t* kv_empty = bars + 18 + C::kStages;   // [kStages]
+    uint64_t* s_free = bars + 18;       // [2]  S has been read into registers (lookahead 2 only)
+    uint64_t* kv_full = bars + 20;                 // [kStages]
+    uint64_t* kv_empty = bars + 20 + C::kStages;   // [kStages]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::kBarriers);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
@@ -244,6 +251,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             mbar_init(&p_full[i], 128);
             mbar_init(&alpha_full[i], 128);
             mbar_init(&final_full[i], 128);
+            mbar_init(&s_free[i], 128);
             mbar_init(&pv_done[i], 1);
             mbar_init(&o_ready[i], 128);
         }
@@ -312,6 +320,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             constexpr uint32_t idesc_o = make_idesc(128, D, 1);
             const uint32_t tS[2] = {tmem_base + C::kColS0, tmem_base + C::kColS1};
             const uint32_t tO[2] = {tmem_base + C::kColO0, tmem_base + C::kColO1};
+            const uint32_t tP[2] = {tmem_base + C::kColP0, tmem_base + C::kColP1};
             uint32_t kv_it = 0;
             uint32_t n_p[2] = {0, 0}, n_or[2] = {0, 0}, n_qf[2] = {0, 0};
             // descriptor words: Q and K tiles are K-major (8-row groups 1024 bytes apart),
@@ -348,8 +357,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             };
             auto fire_PV = [&](int i, bool first) {
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) mma_ts64(tO[i], tS[i] + ks * 8, vd[ks], idesc_o, (!first) || ks > 0);
+                for (int ks = 0; ks < 8; ++ks) mma_ts64(tO[i], tP[i] + ks * 8, vd[ks], idesc_o, (!first) || ks > 0);
             };
+            constexpr int LA = C::kLookahead;
+            uint32_t n_sf[2] = {0, 0};
             for (int w = blockIdx.x; w < prm.n_work; w += gridDim.x) {
                 const int qpair = prm.n_qpairs - 1 - w / prm.BH;
                 const int q0 = qpair * 256;
@@ -358,28 +369,40 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 // ring positions of this work item: K_t at kv_it + 2t, V_t at kv_it + 2t + 1
                 auto stage_of = [&](uint32_t it) { return (int)(it % C::kStages); };
                 auto parity_of = [&](uint32_t it) { return (it / C::kStages) & 1u; };
-                // S_i(0)
-                if (!pf_wait(&kv_full[stage_of(kv_it)], parity_of(kv_it), kWaitKVFull, abort_flag)) goto done;
-                for (int i = 0; i < 2; ++i) {
-                    if (Ti[i] == 0) continue;
-                    if (!pf_wait(&q_full[i], n_qf[i] & 1, kWaitQFull, abort_flag)) goto done;
-                    ++n_qf[i];
+                // S_i(u): score product of key tile u for query tile i; with lookahead 2 the S
+                // region must have been read by the weights warps of step u-1 first
+                auto do_S = [&](int i, int u) -> bool {
+                    const uint32_t it_k = kv_it + 2 * u;
+                    if (u == 0) {
+                        if (!pf_wait(&q_full[i], n_qf[i] & 1, kWaitQFull, abort_flag)) return false;
+                        ++n_qf[i];
+                    } else if (LA > 1) {
+                        if (!pf_wait(&s_free[i], n_sf[i] & 1, kWaitSFree, abort_flag)) return false;
+                        ++n_sf[i];
+                    }
                     tc_fence_after();
-                    prep_S(i, stage_of(kv_it));
+                    prep_S(i, stage_of(it_k));
                     fire_S(i);
                     tc_commit(&s_full[i]);
-                    if (Ti[i] == 1) tc_commit(&q_empty[i]);
+                    if (u + 1 == Ti[i]) tc_commit(&q_empty[i]);
+                    return true;
+                };
+                // prologue: S_i(0) .. S_i(LA-1)
+                for (int u = 0; u < LA && u < T; ++u) {
+                    const uint32_t it_k = kv_it + 2 * u;
+                    if (!pf_wait(&kv_full[stage_of(it_k)], parity_of(it_k), kWaitKVFull, abort_flag)) goto done;
+                    for (int i = 0; i < 2; ++i)
+                        if (u < Ti[i] && !do_S(i, u)) goto done;
+                    tc_commit(&kv_empty[stage_of(it_k)]);
                 }
-                tc_commit(&kv_empty[stage_of(kv_it)]);
                 for (int t = 0; t < T; ++t) {
                     const uint32_t it_v = kv_it + 2 * t + 1;
-                    const uint32_t it_kn = kv_it + 2 * t + 2;
+                    const uint32_t it_kn = kv_it + 2 * (t + LA);
                     if (!pf_wait(&kv_full[stage_of(it_v)], parity_of(it_v), kWaitKVFull, abort_flag)) goto done;
                     bool kn_ready = false;
                     for (int i = 0; i < 2; ++i) {
-                        if (t < Ti[i]) prep_PV(stage_of(it_v));
-                        if (t + 1 < Ti[i]) prep_S(i, stage_of(it_kn));
                         if (t < Ti[i]) {
+                            prep_PV(stage_of(it_v));
                             if (!pf_wait(&p_full[i], n_p[i] & 1, kWaitPFull, abort_flag)) goto done;
                             ++n_p[i];
                             if (!pf_wait(&o_ready[i], n_or[i] & 1, kWaitOReady, abort_flag)) goto done;
@@ -388,19 +411,16 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                             fire_PV(i, t == 0);
                             tc_commit(&pv_done[i]);
                         }
-                        if (t + 1 < Ti[i]) {
+                        if (t + LA < Ti[i]) {
                             if (!kn_ready) {
                                 if (!pf_wait(&kv_full[stage_of(it_kn)], parity_of(it_kn), kWaitKVFull, abort_flag)) goto done;
                                 kn_ready = true;
-                                tc_fence_after();
                             }
-                            fire_S(i);
-                            tc_commit(&s_full[i]);
-                            if (t + 2 == Ti[i]) tc_commit(&q_empty[i]);
+                            if (!do_S(i, t + LA)) goto done;
                         }
                     }
                     tc_commit(&kv_empty[stage_of(it_v)]);
-                    if (t + 1 < T) tc_commit(&kv_empty[stage_of(it_kn)]);
+                    if (t + LA < T) tc_commit(&kv_empty[stage_of(it_kn)]);
                 }
                 kv_it += 2 * T;
             }
@@ -412,8 +432,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const int row = threadIdx.x & 127;             // row within the tile = tensor-memory lane
         const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tS = tmem_base + (i == 0 ? C::kColS0 : C::kColS1) + lane_sel;
+        const uint32_t tP = tmem_base + (i == 0 ? C::kColP0 : C::kColP1) + lane_sel;
         const float c = prm.scale_log2e;
-        uint32_t n_s = 0, n_ae = 0;
+        uint32_t n_s = 0, n_ae = 0, n_pk = 0;
         for (int w = blockIdx.x; w < prm.n_work; w += gridDim.x) {
             const int qpair = prm.n_qpairs - 1 - w / prm.BH;
             const int bh = w % prm.BH;
@@ -431,6 +452,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll
                 for (int cb = 0; cb < 4; ++cb) tmem_ld32(tS + cb * 32, reinterpret_cast<uint32_t*>(s) + cb * 32);
                 tc_wait_ld();
+                if (C::kLookahead > 1 && t + 1 < Ti) {
+                    // S is in registers: the score product of the next step may overwrite it
+                    tc_fence_before();
+                    mbar_arrive(&s_free[i]);
+                }
                 const int n0 = t * 128;
                 if (n0 + 128 > Nk || (prm.causal && n0 + 127 > q0)) {
 #pragma unroll
@@ -471,8 +497,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         pk[j / 2] = pack_bf16x2(p0, p1);
                         pk[j / 2 + 1] = pack_bf16x2(p2, p3);
                     }
-                    tmem_st32(tS + 32 * h, pk);
+                    if (C::kLookahead > 1 && h == 0 && n_pk > 0) {
+                        // P has a region of its own: the previous P V must have read it
+                        if (!pf_wait(&pv_done[i], (n_pk - 1) & 1, kWaitPVDone, abort_flag)) goto done;
+                        tc_fence_after();
+                    }
+                    tmem_st32(tP + 32 * h, pk);
                 }
+                ++n_pk;
                 float a0, a1, a2, a3;
                 unpack2(acc0, a0, a1);
                 unpack2(acc1, a2, a3);
