@@ -335,22 +335,24 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             // products are therefore built while the thread would wait anyway (prep_*), and the
             // products themselves are issued back to back from registers (fire_*).
             constexpr int KS = D / 16;
-            uint64_t qd[KS], kd[KS], vd[8];
-            auto prep_S = [&](int i, int stage) {
-                const uint32_t qa = q_lo[i];
+            uint64_t qd0[KS], qd1[KS], kd[KS], vd[8];
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                const uint32_t off = ((ks >> 2) * C::kPanelBytes + (ks & 3) * 32) >> 4;
+                qd0[ks] = desc64(q_lo[0] + off, desc_hi);
+                qd1[ks] = desc64(q_lo[1] + off, desc_hi);
+            }
+            auto prep_K = [&](int stage) {
                 const uint32_t ka = k_lo0 + stage * (C::kTileBytes >> 4);
 #pragma unroll
-                for (int ks = 0; ks < KS; ++ks) {
-                    const uint32_t off = ((ks >> 2) * C::kPanelBytes + (ks & 3) * 32) >> 4;
-                    qd[ks] = desc64(qa + off, desc_hi);
-                    kd[ks] = desc64(ka + off, desc_hi);
-                }
+                for (int ks = 0; ks < KS; ++ks)
+                    kd[ks] = desc64(ka + (((ks >> 2) * C::kPanelBytes + (ks & 3) * 32) >> 4), desc_hi);
             };
             auto fire_S = [&](int i) {
 #pragma unroll
-                for (int ks = 0; ks < KS; ++ks) mma_ss64(tS[i], qd[ks], kd[ks], idesc_s, ks > 0);
+                for (int ks = 0; ks < KS; ++ks) mma_ss64(tS[i], i == 0 ? qd0[ks] : qd1[ks], kd[ks], idesc_s, ks > 0);
             };
-            auto prep_PV = [&](int stage) {
+            auto prep_V = [&](int stage) {
                 const uint32_t va = v_lo0 + stage * (C::kTileBytes >> 4);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) vd[ks] = desc64(va + ks * (2048 >> 4), desc_hi);   // 16 keys = two 1024-byte atoms
@@ -372,7 +374,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 // S_i(u): score product of key tile u for query tile i; with lookahead 2 the S
                 // region must have been read by the weights warps of step u-1 first
                 auto do_S = [&](int i, int u) -> bool {
-                    const uint32_t it_k = kv_it + 2 * u;
                     if (u == 0) {
                         if (!pf_wait(&q_full[i], n_qf[i] & 1, kWaitQFull, abort_flag)) return false;
                         ++n_qf[i];
@@ -381,7 +382,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         ++n_sf[i];
                     }
                     tc_fence_after();
-                    prep_S(i, stage_of(it_k));
                     fire_S(i);
                     tc_commit(&s_full[i]);
                     if (u + 1 == Ti[i]) tc_commit(&q_empty[i]);
@@ -390,6 +390,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 // prologue: S_i(0) .. S_i(LA-1)
                 for (int u = 0; u < LA && u < T; ++u) {
                     const uint32_t it_k = kv_it + 2 * u;
+                    prep_K(stage_of(it_k));
                     if (!pf_wait(&kv_full[stage_of(it_k)], parity_of(it_k), kWaitKVFull, abort_flag)) goto done;
                     for (int i = 0; i < 2; ++i)
                         if (u < Ti[i] && !do_S(i, u)) goto done;
@@ -398,11 +399,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 for (int t = 0; t < T; ++t) {
                     const uint32_t it_v = kv_it + 2 * t + 1;
                     const uint32_t it_kn = kv_it + 2 * (t + LA);
+                    prep_V(stage_of(it_v));
+                    if (t + LA < T) prep_K(stage_of(it_kn));
                     if (!pf_wait(&kv_full[stage_of(it_v)], parity_of(it_v), kWaitKVFull, abort_flag)) goto done;
                     bool kn_ready = false;
                     for (int i = 0; i < 2; ++i) {
                         if (t < Ti[i]) {
-                            prep_PV(stage_of(it_v));
                             if (!pf_wait(&p_full[i], n_p[i] & 1, kWaitPFull, abort_flag)) goto done;
                             ++n_p[i];
                             if (!pf_wait(&o_ready[i], n_or[i] & 1, kWaitOReady, abort_flag)) goto done;
