@@ -477,9 +477,15 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 }
                 const float ref = fmaxf(L, m0 * c);
                 const float e_old = ex2(L - ref);            // 0 for the first tile (L = -inf), else usually 1
-                if (t > 0) {
-                    // beta = e_old / l_{t-1}: closes step t-1 (its division) and opens step t
-                    sAlpha[(n_ae & 1) * 256 + i * 128 + row] = e_old * inv_l;
+                // beta = e_old / l_{t-1}: closes step t-1 (its division) and opens step t.
+                // The hand-off has no back-pressure barrier, so message n+1 may only be posted
+                // once message n is known to be consumed.  With lookahead 1 that follows from
+                // the order of the products (S(t) is issued after P V(t-1), which needed the
+                // correction of step t-1).  With lookahead 2 S(t) runs ahead, so the message is
+                // posted below, after the wait for P V(t-1) that the P store needs anyway.
+                const float beta = e_old * inv_l;
+                if (C::kLookahead == 1 && t > 0) {
+                    sAlpha[(n_ae & 1) * 256 + i * 128 + row] = beta;
                     ++n_ae;
                     mbar_arrive(&alpha_full[i]);
                 }
@@ -503,6 +509,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         // P has a region of its own: the previous P V must have read it
                         if (!pf_wait(&pv_done[i], (n_pk - 1) & 1, kWaitPVDone, abort_flag)) goto done;
                         tc_fence_after();
+                        if (t > 0) {
+                            sAlpha[(n_ae & 1) * 256 + i * 128 + row] = beta;
+                            ++n_ae;
+                            mbar_arrive(&alpha_full[i]);
+                        }
                     }
                     tmem_st32(tP + 32 * h, pk);
                 }
@@ -518,7 +529,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 mbar_arrive(&p_full[i]);
             }
             if (Ti > 0) {
-                // the reciprocal that closes the last step goes to the epilogue
+                // the reciprocal that closes the last step goes to the epilogue.  The previous
+                // work item's message must have been consumed: for items of two or more tiles
+                // that follows from the product order; a one-tile item waits for its own P V,
+                // which is issued only after the previous epilogue has released O.
+                if (Ti == 1 && !pf_wait(&pv_done[i], (n_pk - 1) & 1, kWaitPVDone, abort_flag)) goto done;
                 sFinal[i * 128 + row] = inv_l;
                 mbar_arrive(&final_full[i]);
             }
