@@ -31,6 +31,10 @@ L2_BYTES = 126e6
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (c4: a batch-4 capture scaled by 16, traffic being
+# proportional to the bytes streamed).  Must be set back to None when that kernel changes.
+NCU_TRAFFIC_BYTES = {"c1": 38.1e6, "c2": 585.4e6, "c3": None, "c4": 34.49e9}
 
 
 def f32(x: float) -> float:
@@ -408,13 +412,15 @@ def main():
         alg = w.kv_bytes
         achieved = alg / (local_ms / args.steps * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if args.batch == 0 else None,
+                "peak_source": peaks["source"],
                 "frac_of_nominal": achieved / NOMINAL_HBM_GBS,
                 "kernel": "splitk_partial_kernel (+combine, timed together)"}
     else:
         achieved = w.flops / (local_ms / args.steps * 1e-3) / 1e12
         roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["bf16_tflops"], "traffic": None, "peak_source": peaks["source"],
+                "frac": achieved / peaks["bf16_tflops"], "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if args.batch == 0 else None,
+                "peak_source": peaks["source"],
                 "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS, "kernel": f"prefill_kernel<{w.d}>"}
 
     line = {
