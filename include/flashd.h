@@ -57,15 +57,18 @@ typedef enum { FLASHD_BF16 = 0, FLASHD_F32 = 1 } flashd_dtype;
 /* ------------------------------------------------------------------------
  * Tiled tensor-core forward (bf16 in, fp32 accumulate, bf16 out).
  *
- * Computes Algorithm 3 with keys grouped in tiles of 128: for each tile the
- * weights of its keys and the weight (1 - W) of the old output follow from
- * Eq. (w-last) applied to the tile as one "super-key" whose score is the
- * log-sum-exp L_T of the tile's scores:
- *     L_new = L_T - ln sigma(L_T - L_old),  P_j = exp(s_j - L_new),
- *     alpha = exp(L_old - L_new),           O <- alpha O + P V_tile,
- * which is Eq. (out-final) for the group.  The carried state per query row is
- * L alone (= s_i - ln w_i of the paper).  S = Q K^T and P V run on the 5th
- * generation tensor cores (tcgen05.mma, accumulators in tensor memory).
+ * Computes Algorithm 3 with keys grouped in tiles of 128.  With x_j = s_j - L_old
+ * and L = s - ln w the carried state, the per-key step of Eq. (w-last) and
+ * Eq. (out-final) with its division written out, o = (o_old + e^x v)/(1 + e^x),
+ * becomes for a tile
+ *     O_new = (O_old + sum_j e^{x_j} v_j) / (1 + sum_j e^{x_j}),
+ *     L_new = L_old + ln(1 + sum_j e^{x_j}),
+ * evaluated relative to a tile-local reference max(L_old, max_j s_j) so that no
+ * exponent is positive.  The reciprocal that closes a tile step is applied when
+ * the next step opens (the last one when the result is stored); no running
+ * maximum and no separate softmax denominator are carried.  S = Q K^T and P V
+ * run on the 5th generation tensor cores (tcgen05.mma, accumulators in tensor
+ * memory).
  *
  * q, o: [B,H,Nq,d] bf16; k, v: [B,H,Nk,d] bf16.  d must be 64 or 128.
  * o must not overlap q, k or v.  Returns after the launch.               */
