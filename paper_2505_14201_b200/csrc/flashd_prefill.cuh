@@ -465,15 +465,23 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     for (int j = 0; j < 128; ++j) s[j] = (n0 + j < limit) ? s[j] : (c >= 0.f ? -INFINITY : INFINITY);
                 }
                 // tile-local reference: max over {L_{t-1}, c*s_j}
-                float m0 = s[0], m1 = s[1];
+                float m0 = s[0], m1 = s[1], m2 = s[2], m3 = s[3];     // four chains: short dependent latency
                 if (c >= 0.f) {
 #pragma unroll
-                    for (int j = 2; j < 126; j += 4) { m0 = max3(m0, s[j], s[j + 1]); m1 = max3(m1, s[j + 2], s[j + 3]); }
-                    m0 = max3(m0, m1, fmaxf(s[126], s[127]));
+                    for (int j = 4; j < 124; j += 8) {
+                        m0 = max3(m0, s[j], s[j + 1]); m1 = max3(m1, s[j + 2], s[j + 3]);
+                        m2 = max3(m2, s[j + 4], s[j + 5]); m3 = max3(m3, s[j + 6], s[j + 7]);
+                    }
+                    m0 = max3(m0, s[124], s[125]); m1 = max3(m1, s[126], s[127]);
+                    m0 = fmaxf(max3(m0, m1, m2), m3);
                 } else {
 #pragma unroll
-                    for (int j = 2; j < 126; j += 4) { m0 = min3(m0, s[j], s[j + 1]); m1 = min3(m1, s[j + 2], s[j + 3]); }
-                    m0 = min3(m0, m1, fminf(s[126], s[127]));
+                    for (int j = 4; j < 124; j += 8) {
+                        m0 = min3(m0, s[j], s[j + 1]); m1 = min3(m1, s[j + 2], s[j + 3]);
+                        m2 = min3(m2, s[j + 4], s[j + 5]); m3 = min3(m3, s[j + 6], s[j + 7]);
+                    }
+                    m0 = min3(m0, s[124], s[125]); m1 = min3(m1, s[126], s[127]);
+                    m0 = fminf(min3(m0, m1, m2), m3);
                 }
                 const float ref = fmaxf(L, m0 * c);
                 const float e_old = ex2(L - ref);            // 0 for the first tile (L = -inf), else usually 1
