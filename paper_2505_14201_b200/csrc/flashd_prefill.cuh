@@ -270,6 +270,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
     const int Nq = prm.Nq, Nk = prm.Nk;
     const int n_kt_all = (Nk + 127) >> 7;
+    // Work items are ordered heaviest first (late query tiles when causal) and dealt to the
+    // CTAs in snake order: round n goes 0..G-1 when n is even and G-1..0 when n is odd, which
+    // evens out the per-CTA totals of a descending cost sequence without a dynamic scheduler.
+    auto work_index = [&](int n) -> int {
+        const int g = (int)gridDim.x, k = (int)blockIdx.x;
+        return n * g + ((n & 1) ? g - 1 - k : k);
+    };
     // key tiles needed by query tile i (rows q0 .. q0+127) of a work item; 0 if the tile is empty
     auto n_tiles = [&](int q0) -> int {
         if (q0 >= Nq) return 0;
@@ -284,7 +291,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         if (lane == 0) {
             uint32_t kv_it = 0;
             uint32_t n_q[2] = {0, 0};     // uses of each Q buffer so far
-            for (int w = blockIdx.x; w < prm.n_work; w += gridDim.x) {
+            for (int nw = 0, w = work_index(0); w < prm.n_work; w = work_index(++nw)) {
                 const int qpair = prm.n_qpairs - 1 - w / prm.BH;
                 const int bh = w % prm.BH;
                 const int q0 = qpair * 256;
@@ -363,7 +370,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             };
             constexpr int LA = C::kLookahead;
             uint32_t n_sf[2] = {0, 0};
-            for (int w = blockIdx.x; w < prm.n_work; w += gridDim.x) {
+            for (int nw = 0, w = work_index(0); w < prm.n_work; w = work_index(++nw)) {
                 const int qpair = prm.n_qpairs - 1 - w / prm.BH;
                 const int q0 = qpair * 256;
                 const int Ti[2] = {n_tiles(q0), n_tiles(q0 + 128)};
@@ -437,7 +444,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const uint32_t tP = tmem_base + (i == 0 ? C::kColP0 : C::kColP1) + lane_sel;
         const float c = prm.scale_log2e;
         uint32_t n_s = 0, n_ae = 0, n_pk = 0;
-        for (int w = blockIdx.x; w < prm.n_work; w += gridDim.x) {
+        for (int nw = 0, w = work_index(0); w < prm.n_work; w = work_index(++nw)) {
             const int qpair = prm.n_qpairs - 1 - w / prm.BH;
             const int bh = w % prm.BH;
             const int q0 = qpair * 256 + i * 128;
@@ -554,7 +561,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tO[2] = {tmem_base + C::kColO0 + lane_sel, tmem_base + C::kColO1 + lane_sel};
         uint32_t n_af[2] = {0, 0}, n_pv[2] = {0, 0}, n_fin[2] = {0, 0};
-        for (int w = blockIdx.x; w < prm.n_work; w += gridDim.x) {
+        for (int nw = 0, w = work_index(0); w < prm.n_work; w = work_index(++nw)) {
             const int qpair = prm.n_qpairs - 1 - w / prm.BH;
             const int bh = w % prm.BH;
             const int q0 = qpair * 256;
