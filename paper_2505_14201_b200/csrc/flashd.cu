@@ -354,6 +354,20 @@ int flashd_attn_fwd_host(const void* q, const void* k, const void* v, void* o, i
         splits = flashd_splitk_num_splits(B, H, Nq, Nk, d);
         wsb = flashd_splitk_workspace_bytes(B, H, Nq, d, splits);
     }
+    // keep freed staging buffers in the device's default pool instead of returning them to
+    // the driver at every synchronisation (set once per device)
+    {
+        static bool pool_set[64] = {false};
+        int dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64 && !pool_set[dev]) {
+            cudaMemPool_t pool;
+            if (cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess) {
+                unsigned long long keep = ~0ull;
+                cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+            }
+            pool_set[dev] = true;
+        }
+    }
     void *dq = nullptr, *dk = nullptr, *dv = nullptr, *dout = nullptr, *dws = nullptr;
     int st = FLASHD_OK;
     bool ok = cudaMallocAsync(&dq, qb, s) == cudaSuccess && cudaMallocAsync(&dk, kb, s) == cudaSuccess &&
