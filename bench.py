@@ -334,6 +334,30 @@ def bench_e2e(fd, w, steps, warmup, torch):
             "workload": w.name}
 
 
+def run_skip_stats(fd, synth, torch, device):
+    """The paper's second experiment in shape: share of output updates that the static range
+    rule [-6, 11] on s_i - s_{i-1} (and the adaptive reading on the sigmoid argument, [-6, 6])
+    would bypass, on the synthetic workloads (config 4 on its first 4 batch elements)."""
+    import dataclasses
+    out = {}
+    for name in ("c0", "c1", "c2", "c3", "c4"):
+        w = synth.WORKLOADS[name]
+        if name == "c4":
+            w = dataclasses.replace(w, B=4)
+        q, k, _ = synth.make_inputs(w, device=device)
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        c = fd.flashd_skip_stats(q, k, f32(w.scale), w.causal)
+        e1.record(); torch.cuda.synchronize()
+        out[name] = {"steps": c[0], "static_keep_pct": 100.0 * c[1] / c[0], "static_replace_pct": 100.0 * c[2] / c[0],
+                     "static_total_pct": 100.0 * (c[1] + c[2]) / c[0], "adaptive_keep_pct": 100.0 * c[3] / c[0],
+                     "adaptive_replace_pct": 100.0 * c[4] / c[0], "ms": e0.elapsed_time(e1)}
+        del q, k
+        torch.cuda.empty_cache()
+    print(json.dumps({"metric": "bypassable_output_updates_pct", "static_range": [-6, 11], "adaptive_range": [-6, 6],
+                      "data": "synthetic", "workloads": out}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -343,6 +367,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the other configurations and the CPU baseline")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--skip-stats", action="store_true",
+                    help="print the bypassable-update statistic (Sec. III-C / V-B) of every workload instead of timing")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the workload's batch size B (smaller case for profiler captures)")
     args = ap.parse_args()
@@ -371,6 +397,10 @@ def main():
     if args.batch > 0:
         import dataclasses
         w = dataclasses.replace(w, B=args.batch, name=f"{w.name} (B={args.batch})")
+
+    if args.skip_stats:
+        run_skip_stats(fd, synth, torch, device)
+        return
 
     sampler = ClockSampler(local_rank)
     # ---- headline: device-resident inputs

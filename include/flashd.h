@@ -178,6 +178,26 @@ int flashd_attn_fwd_splitk_static(const void* q, const void* k, const void* v, v
                                   int num_splits, void* stream);
 
 /* ------------------------------------------------------------------------
+ * Bypassable-update statistic (Sec. III-C, Sec. V-B, Table I).
+ *
+ * Walks every query over its visible keys as Algorithm 3 does (state
+ * s_{i-1}, ln w_{i-1}; no output is formed) and counts, over all steps i >= 2,
+ *   counts[0]  steps examined
+ *   counts[1]  s_i - s_{i-1} <= lo   (static criterion: w_i ~ 0, update bypassed)
+ *   counts[2]  s_i - s_{i-1} >= hi   (static criterion: w_i ~ 1, output replaced)
+ *   counts[3]  x_i <= alo            x_i = s_i - s_{i-1} + ln w_{i-1}, the sigmoid
+ *   counts[4]  x_i >= ahi            argument of Eq. (w-last)
+ * The paper uses [lo, hi] = [-6, 11]; [alo, ahi] is this library's reading of
+ * the adaptive criterion the paper leaves to future work ([-6, 6] suits the
+ * unshifted sigmoid).  Scores and the decisions are taken in fp64.
+ * counts: DEVICE pointer to 5 unsigned 64-bit integers, 8-byte aligned; the
+ * call zeroes them on `stream` before the kernel adds to them.
+ * in_dtype FLASHD_BF16 or FLASHD_F32; d in {32, 64, 128, 256}.               */
+int flashd_skip_stats(const void* q, const void* k, unsigned long long* counts, int in_dtype,
+                      int B, int H, int Nq, int Nk, int d, float scale, int causal,
+                      float lo, float hi, float alo, float ahi, void* stream);
+
+/* ------------------------------------------------------------------------
  * End-to-end call on HOST buffers: q, k, v, o are host pointers (pinned
  * memory gives asynchronous copies).  The call allocates device buffers from
  * the stream-ordered pool of the current device, copies q, k, v in, runs the

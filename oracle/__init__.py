@@ -57,7 +57,7 @@ def _load():
             lib.oracle_attn_tiled.argtypes = [_D, _D, _D, _D, _D, _D, _D, ci, ci, ci, ci, ci, cd, ci, _I, ci, ci]
             lib.oracle_split_merge.argtypes = [_D, _D, _D, _D, ci, ci, ci]
             lib.oracle_flashd_weights.argtypes = [_D, ci, _D, ci]
-            lib.oracle_skip_stats.argtypes = [_D, _D, _LL, ci, ci, ci, ci, ci, cd, ci, _I, cd, cd]
+            lib.oracle_skip_stats.argtypes = [_D, _D, _LL, ci, ci, ci, ci, ci, cd, ci, _I, cd, cd, cd, cd, cd]
             for f in ("oracle_attn_naive", "oracle_attn_alg1", "oracle_attn_alg2",
                       "oracle_attn_flashd", "oracle_attn_tiled", "oracle_split_merge",
                       "oracle_flashd_weights", "oracle_skip_stats"):
@@ -194,13 +194,16 @@ def flashd_weights(s, variant=0):
     return w
 
 
-def skip_stats(q, k, scale, causal=False, q_index=None, lo=-6.0, hi=11.0):
-    """Static criterion of Sec. III-C: (steps, diffs <= lo, diffs >= hi)."""
+def skip_stats(q, k, scale, causal=False, q_index=None, lo=-6.0, hi=11.0, alo=-6.0, ahi=6.0, near=1e-4):
+    """Bypassable output updates (Sec. III-C / V-B).  Returns (steps, diff <= lo,
+    diff >= hi, x <= alo, x >= ahi, steps within ``near`` of a threshold) where
+    diff = s_i - s_{i-1} and x = diff + ln w_{i-1}."""
     q, k = _f64(q), _f64(k)
     B, H, Nq, d = q.shape
     Nk = k.shape[2]
     qi = None if q_index is None else np.ascontiguousarray(np.asarray(q_index, dtype=np.int32))
-    counts = np.zeros(3, dtype=np.int64)
+    counts = np.zeros(6, dtype=np.int64)
     _load().oracle_skip_stats(_p(q), _p(k), counts.ctypes.data_as(_LL), B, H, Nq, Nk, d,
-                              float(scale), int(bool(causal)), _pi(qi), float(lo), float(hi))
+                              float(scale), int(bool(causal)), _pi(qi), float(lo), float(hi),
+                              float(alo), float(ahi), float(near))
     return tuple(int(c) for c in counts)

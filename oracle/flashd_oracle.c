@@ -386,33 +386,53 @@ void oracle_split_merge(const double* partial_o, const double* partial_L,
 }
 
 /* ------------------------------------------------------------------------ */
-/* Sec. III-C / Sec. V-B: the static criterion.  For every query and every
- * visible key after the first, count the steps whose score difference
- * s_i - s_{i-1} lies outside [lo, hi] (the paper uses [-6, 11]); these are the
- * output updates the paper proposes to bypass.  counts[0] = steps examined,
- * counts[1] = differences <= lo, counts[2] = differences >= hi.            */
+/* Sec. III-C / Sec. V-B: how often an output update could be bypassed.
+ * Static criterion (the paper's): for every query and every visible key after
+ * the first, the step is counted when the score difference s_i - s_{i-1} is
+ * <= lo (w_i ~ 0, output kept) or >= hi (w_i ~ 1, output replaced); the paper
+ * uses [lo, hi] = [-6, 11].
+ * Adaptive criterion: Sec. V-B only announces "an adaptive criterion that
+ * includes both the range of attention score differences and the value of the
+ * previous weight".  Reading taken here: the same test applied to the actual
+ * sigmoid argument of Eq. (w-last), x_i = s_i - s_{i-1} + ln w_{i-1}, with its
+ * own thresholds [alo, ahi] (for the unshifted sigmoid the paper's figure
+ * suggests [-6, 6]).
+ * counts[0] steps examined, [1] differences <= lo, [2] differences >= hi,
+ * [3] x <= alo, [4] x >= ahi, [5] steps within `near` of any of the four
+ * thresholds (so that a comparison with another implementation can tell a
+ * rounding tie from a mistake).                                             */
 void oracle_skip_stats(const double* q, const double* k, long long* counts,
                        int B, int H, int Nq, int Nk, int d,
                        double scale, int causal, const int* q_index,
-                       double lo, double hi) {
-    long long total = 0, below = 0, above = 0;
+                       double lo, double hi, double alo, double ahi, double near) {
+    long long total = 0, below = 0, above = 0, abelow = 0, aabove = 0, nnear = 0;
     for (int bh = 0; bh < B * H; ++bh) {
         for (int i = 0; i < Nq; ++i) {
             const double* qi = q + ((size_t)bh * Nq + i) * d;
             const double* kb = k + (size_t)bh * Nk * d;
             int nv = n_visible(q_global(q_index, i), Nk, causal);
-            double s_prev = 0.0;
+            double s_prev = 0.0, lnw = 0.0;
             for (int j = 0; j < nv; ++j) {
                 double s = dot_scaled(qi, kb + (size_t)j * d, d, scale);
                 if (j > 0) {
                     double diff = s - s_prev;
+                    double x = diff + lnw;             /* argument of Eq. (w-last) */
                     ++total;
                     if (diff <= lo) ++below;
                     else if (diff >= hi) ++above;
+                    if (x <= alo) ++abelow;
+                    else if (x >= ahi) ++aabove;
+                    if (fabs(diff - lo) < near || fabs(diff - hi) < near ||
+                        fabs(x - alo) < near || fabs(x - ahi) < near) ++nnear;
+                    double w;
+                    flashd_weight_step(0, s, s_prev, lnw, &w, &lnw);
+                } else {
+                    lnw = 0.0;
                 }
                 s_prev = s;
             }
         }
     }
     counts[0] = total; counts[1] = below; counts[2] = above;
+    counts[3] = abelow; counts[4] = aabove; counts[5] = nnear;
 }

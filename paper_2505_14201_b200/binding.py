@@ -18,7 +18,7 @@ EXPORTED_SYMBOLS = (
     "flashd_attn_fwd", "flashd_attn_fwd_ex", "flashd_attn_fwd_f32", "flashd_attn_fwd_perkey",
     "flashd_splitk_workspace_bytes", "flashd_splitk_num_splits", "flashd_splitk_partial",
     "flashd_splitk_combine", "flashd_attn_fwd_splitk", "flashd_attn_fwd_splitk_static",
-    "flashd_attn_fwd_host", "flashd_last_device_status", "flashd_status_string", "flashd_version", "flashd_launch_count",
+    "flashd_attn_fwd_host", "flashd_skip_stats", "flashd_last_device_status", "flashd_status_string", "flashd_version", "flashd_launch_count",
 )
 
 _lock = threading.Lock()
@@ -60,6 +60,7 @@ def lib() -> ctypes.CDLL:
             L.flashd_splitk_combine.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, vp]
             L.flashd_attn_fwd_splitk.argtypes = [vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_attn_fwd_splitk_static.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, ci, vp]
+            L.flashd_skip_stats.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, cf, cf, cf, cf, vp]
             L.flashd_attn_fwd_host.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
             L.flashd_status_string.argtypes = [ci]
@@ -253,6 +254,22 @@ def flashd_attn_fwd_host(q, k, v, scale, causal=False, path=0, o=None, stream=No
     _check(lib().flashd_attn_fwd_host(_ptr(q), _ptr(k), _ptr(v), _ptr(o), int(path), B, H, Nq, Nk, d,
                                       float(scale), int(bool(causal)), _stream_ptr(stream)), "flashd_attn_fwd_host")
     return o
+
+
+def flashd_skip_stats(q, k, scale, causal=False, lo=-6.0, hi=11.0, alo=-6.0, ahi=6.0, stream=None):
+    """Bypassable-update counts (steps, diff <= lo, diff >= hi, x <= alo, x >= ahi) as Python ints."""
+    import torch
+    if q.dim() != 4 or k.dim() != 4 or q.shape[:2] != k.shape[:2] or q.shape[3] != k.shape[3]:
+        raise ValueError("q, k must be [B, H, N, d] with matching B, H, d")
+    if not (q.is_contiguous() and k.is_contiguous()):
+        raise ValueError("q, k must be contiguous")
+    B, H, Nq, d = q.shape
+    Nk = k.shape[2]
+    counts = torch.empty(5, dtype=torch.int64, device=q.device)
+    _check(lib().flashd_skip_stats(_ptr(q), _ptr(k), _ptr(counts), _dtype_code(q), B, H, Nq, Nk, d, float(scale),
+                                   int(bool(causal)), float(lo), float(hi), float(alo), float(ahi),
+                                   _stream_ptr(stream)), "flashd_skip_stats")
+    return tuple(int(x) for x in counts.cpu().tolist())
 
 
 def flashd_last_device_status(stream=None):

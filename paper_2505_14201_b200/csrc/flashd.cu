@@ -14,6 +14,7 @@
 #include "flashd_decode.cuh"
 #include "flashd_perkey.cuh"
 #include "flashd_prefill.cuh"
+#include "flashd_skipstats.cuh"
 
 namespace {
 
@@ -336,6 +337,43 @@ int flashd_attn_fwd_splitk_static(const void* q, const void* k, const void* v, v
     __nv_bfloat16* out = static_cast<__nv_bfloat16*>(o);
     if (d == 128) splitk_combine_kernel<128, __nv_bfloat16><<<(unsigned)rows, 128, 0, s>>>(ws, out, nullptr, num_splits);
     else splitk_combine_kernel<64, __nv_bfloat16><<<(unsigned)rows, 64, 0, s>>>(ws, out, nullptr, num_splits);
+    return after_launch();
+}
+
+int flashd_skip_stats(const void* q, const void* k, unsigned long long* counts, int in_dtype, int B, int H, int Nq,
+                      int Nk, int d, float scale, int causal, float lo, float hi, float alo, float ahi,
+                      void* stream) {
+    if (!q || !k || !counts) return FLASHD_ERR_NULL;
+    if (B <= 0 || H <= 0 || Nq <= 0 || Nk <= 0 || d <= 0 || !std::isfinite(scale)) return FLASHD_ERR_SHAPE;
+    if (!(lo <= hi) || !(alo <= ahi)) return FLASHD_ERR_SHAPE;
+    if (!aligned16(q) || !aligned16(k) || (reinterpret_cast<uintptr_t>(counts) & 7u)) return FLASHD_ERR_ALIGN;
+    if (d != 32 && d != 64 && d != 128 && d != 256) return FLASHD_ERR_UNSUPPORTED;
+    if (in_dtype != FLASHD_BF16 && in_dtype != FLASHD_F32) return FLASHD_ERR_UNSUPPORTED;
+    const long long rows = (long long)B * H * Nq;
+    const int warps = 4;
+    const long long blocks = (rows + warps - 1) / warps;
+    if (blocks > 0x7fffffffLL) return FLASHD_ERR_SHAPE;
+    cudaStream_t s = as_stream(stream);
+    if (cudaMemsetAsync(counts, 0, 5 * sizeof(unsigned long long), s) != cudaSuccess) return FLASHD_ERR_CUDA;
+#define FLASHD_LAUNCH_STATS(T, E) \
+    skipstats_kernel<T, E><<<(unsigned)blocks, warps * 32, 0, s>>>(static_cast<const T*>(q), static_cast<const T*>(k), \
+                                                                  counts, rows, Nq, Nk, scale, causal, lo, hi, alo, ahi)
+    if (in_dtype == FLASHD_BF16) {
+        switch (d) {
+            case 32: FLASHD_LAUNCH_STATS(__nv_bfloat16, 1); break;
+            case 64: FLASHD_LAUNCH_STATS(__nv_bfloat16, 2); break;
+            case 128: FLASHD_LAUNCH_STATS(__nv_bfloat16, 4); break;
+            default: FLASHD_LAUNCH_STATS(__nv_bfloat16, 8); break;
+        }
+    } else {
+        switch (d) {
+            case 32: FLASHD_LAUNCH_STATS(float, 1); break;
+            case 64: FLASHD_LAUNCH_STATS(float, 2); break;
+            case 128: FLASHD_LAUNCH_STATS(float, 4); break;
+            default: FLASHD_LAUNCH_STATS(float, 8); break;
+        }
+    }
+#undef FLASHD_LAUNCH_STATS
     return after_launch();
 }
 

@@ -379,16 +379,32 @@ def test_linear_domain_weight_freezes_after_underflow():
 # skip statistic (Sec. III-C static range): brute-force count
 # --------------------------------------------------------------------------
 def test_skip_stats_counts():
+    """Static and adaptive counts against a plain Python count; the adaptive
+    argument uses the closed form ln w_{i-1} = s_{i-1} - ln sum_{j<i} e^{s_j}
+    (Eq. w-basic) instead of the oracle's recurrence."""
     rng = np.random.default_rng(77)
     B, H, Nq, Nk, d = 1, 2, 5, 9, 3
     q = rng.normal(size=(B, H, Nq, d)) * 4; k = rng.normal(size=(B, H, Nk, d)) * 4
     for causal in (False, True):
-        total = below = above = 0
+        total = below = above = abelow = aabove = 0
         for b, h, i in itertools.product(range(B), range(H), range(Nq)):
             nv = min(i + 1, Nk) if causal else Nk
             s = [float(np.dot(q[b, h, i], k[b, h, j])) for j in range(nv)]
             for j in range(1, nv):
+                diff = s[j] - s[j - 1]
+                lnw_prev = s[j - 1] - float(scipy.special.logsumexp(s[:j]))
+                x = diff + lnw_prev
                 total += 1
-                below += (s[j] - s[j - 1]) <= -6
-                above += (s[j] - s[j - 1]) >= 11
-        assert oracle.skip_stats(q, k, 1.0, causal) == (total, below, above)
+                below += diff <= -6
+                above += diff >= 11
+                abelow += x <= -6
+                aabove += x >= 6
+        got = oracle.skip_stats(q, k, 1.0, causal)
+        assert got[:5] == (total, below, above, abelow, aabove)
+        assert got[5] == 0
+    # integer scores: thresholds hit exactly, ties count as bypassable
+    qq = np.zeros((1, 1, 1, 2)); qq[0, 0, 0, 0] = 1
+    kk = np.zeros((1, 1, 5, 2)); kk[0, 0, :, 0] = [0, -6, 5, 16, 16]
+    got = oracle.skip_stats(qq, kk, 1.0)
+    assert got[0] == 4 and got[1] == 1 and got[2] == 2     # diffs -6, 11, 11, 0
+    assert got[5] >= 3
