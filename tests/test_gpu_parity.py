@@ -154,6 +154,36 @@ def test_prefill_shapes(flashd_lib, shape):
     assert torch.equal(again, got)
 
 
+@pytest.mark.parametrize("shape", [(2, 200, 100, 100, 64, True), (2, 200, 128, 128, 128, False), (1, 300, 1, 77, 64, False),
+                                   (1, 160, 256, 128, 64, True), (1, 150, 130, 1, 128, False)])
+def test_prefill_many_short_work_items(flashd_lib, shape):
+    """More work items than CTAs, each of one or two key tiles: exercises the hand-offs across
+    work-item boundaries (one-tile items post only the closing reciprocal)."""
+    B, H, Nq, Nk, d, causal = shape
+    q, k, v = synth.random_qkv(B, H, Nq, Nk, d, seed=500 + Nq + Nk)
+    sc = f32_scale(d)
+    want = oracle.attn_naive(q, k, v, sc, causal)
+    qc, kc, vc = q.cuda(), k.cuda(), v.cuda()
+    got = flashd_lib.flashd_attn_fwd(qc, kc, vc, sc, causal)
+    got32 = flashd_lib.flashd_attn_fwd_ex(qc, kc, vc, sc, causal, out_dtype=torch.float32)
+    ok_status(flashd_lib)
+    check_tiled(got, got32, want, shape)
+    for _ in range(5):                     # repeated launches: bit-identical, no stale state
+        assert torch.equal(flashd_lib.flashd_attn_fwd(qc, kc, vc, sc, causal), got)
+    ok_status(flashd_lib)
+
+
+def test_prefill_zero_scale_is_rejected(flashd_lib):
+    q, k, v = synth.random_qkv(1, 1, 8, 8, 64, seed=1, device="cuda")
+    with pytest.raises(flashd_lib.FlashdError) as ei:
+        flashd_lib.flashd_attn_fwd(q, k, v, 0.0, False)
+    assert ei.value.status == 3
+    # the per-key path handles it: equal scores, running mean of V
+    got = flashd_lib.flashd_attn_fwd_perkey(q, k, v, 0.0, False, out_dtype=torch.float32)
+    want = v.float().mean(dim=2, keepdim=True).expand_as(got)
+    assert torch.allclose(got, want, atol=1e-5)
+
+
 def test_prefill_structured_inputs(flashd_lib):
     """Cases whose answer is known without the oracle."""
     B, H, N, d = 1, 2, 384, 128
