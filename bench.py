@@ -358,6 +358,37 @@ def run_skip_stats(fd, synth, torch, device):
                       "data": "synthetic", "workloads": out}), flush=True)
 
 
+def run_gqa(fd, synth, torch, device, peaks, steps):
+    """Grouped-query decode: config 4 with its 32 query heads sharing 32/G K/V heads.  The K/V
+    stream (the algorithmic bytes) shrinks by G, the arithmetic per K/V byte grows by G."""
+    w4 = synth.WORKLOADS["c4"]
+    out = {}
+    for G in (1, 4, 8):
+        Hkv = w4.H // G
+        g = torch.Generator(device=device).manual_seed(w4.seed + G)
+        q = torch.randn(w4.B, w4.H, 1, w4.d, generator=g, device=device).to(torch.bfloat16)
+        k = torch.randn(w4.B, Hkv, w4.Nk, w4.d, generator=g, device=device).to(torch.bfloat16)
+        v = torch.randn(w4.B, Hkv, w4.Nk, w4.d, generator=g, device=device).to(torch.bfloat16)
+        sc = f32(w4.scale)
+        S = fd.flashd_gqa_num_splits(w4.B, Hkv, G, w4.Nk, w4.d)
+        ws = torch.empty((w4.B, w4.H, 1, S, w4.d + 1), dtype=torch.float32, device=device)
+        o = torch.empty_like(q)
+        ms = time_gpu(lambda i: fd.flashd_attn_fwd_gqa(q, k, v, sc, S, workspace=ws, o=o), steps, 3, torch) / steps
+        alg = (k.numel() + v.numel() + q.numel() + o.numel()) * 2
+        flops = 4.0 * w4.B * w4.H * w4.Nk * w4.d
+        out[f"G={G}"] = {"B": w4.B, "Hkv": Hkv, "G": G, "Nk": w4.Nk, "d": w4.d, "num_splits": S, "ms_per_step": ms,
+                         "gbs": alg / (ms * 1e-3) / 1e9, "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                         "frac_hbm_nominal": alg / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+                         "tflops": flops / (ms * 1e-3) / 1e12, "kv_gb": (k.numel() + v.numel()) * 2 / 1e9}
+        del q, k, v, ws, o
+        torch.cuda.empty_cache()
+    st, detail = fd.flashd_last_device_status()
+    if st != 0:
+        raise SystemExit(f"device status {st} {detail}")
+    print(json.dumps({"metric": "gqa_decode_hbm_gbs", "unit": "GB/s", "data": "synthetic", "steps": steps,
+                      "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "groups": out}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -369,6 +400,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--skip-stats", action="store_true",
                     help="print the bypassable-update statistic (Sec. III-C / V-B) of every workload instead of timing")
+    ap.add_argument("--gqa", action="store_true",
+                    help="time the grouped-query decode variant (config 4 with shared K/V heads) instead")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the workload's batch size B (smaller case for profiler captures)")
     args = ap.parse_args()
@@ -400,6 +433,10 @@ def main():
 
     if args.skip_stats:
         run_skip_stats(fd, synth, torch, device)
+        return
+
+    if args.gqa:
+        run_gqa(fd, synth, torch, device, peaks, min(args.steps, 30))
         return
 
     sampler = ClockSampler(local_rank)

@@ -140,6 +140,36 @@ int flashd_attn_fwd_splitk(const void* q, const void* k, const void* v, void* o,
                            int num_splits, void* stream);
 
 /* ------------------------------------------------------------------------
+ * Grouped-query split-K forward (decode with shared K/V heads).
+ * One query position, bf16 in, d = 128 or 64, non-causal.
+ *
+ * G consecutive query heads attend to the same K/V head: query head
+ * h = hkv*G + g reads k[b,hkv], v[b,hkv].  The attention function of every
+ * query head is unchanged (Eq. (out-final)/(w-last) per head); only the data
+ * movement differs: each split's K and V rows are read from device memory
+ * once and serve all G queries.
+ *   q, o : [B, Hkv*G, 1, d] contiguous;  k, v : [B, Hkv, Nk, d] contiguous.
+ *   1 <= G <= FLASHD_MAX_GROUP (larger: FLASHD_ERR_UNSUPPORTED).
+ * flashd_gqa_partial writes the partial states [B, Hkv*G, 1, num_splits, d+1]
+ * fp32 exactly as flashd_splitk_partial does for a [B, Hkv*G, 1, d] query
+ * tensor, so flashd_splitk_combine(workspace, o, lse, B, Hkv*G, 1, d, ...)
+ * finishes it; flashd_attn_fwd_gqa queues both (bf16 output).  Workspace
+ * size: flashd_splitk_workspace_bytes(B, Hkv*G, 1, d, num_splits); ownership,
+ * alignment, split rules and errors as for the split-K calls above.
+ * flashd_gqa_num_splits returns the library's split count (num_splits <= 0
+ * in flashd_attn_fwd_gqa selects it).                                      */
+#define FLASHD_MAX_GROUP 8
+int flashd_gqa_num_splits(int B, int Hkv, int G, int Nk, int d);
+int flashd_gqa_partial(const void* q, const void* k, const void* v,
+                       void* workspace, size_t workspace_bytes,
+                       int B, int Hkv, int G, int Nk, int d, float scale,
+                       int num_splits, void* stream);
+int flashd_attn_fwd_gqa(const void* q, const void* k, const void* v, void* o,
+                        void* workspace, size_t workspace_bytes,
+                        int B, int Hkv, int G, int Nk, int d, float scale,
+                        int num_splits, void* stream);
+
+/* ------------------------------------------------------------------------
  * Split-K forward that allocates nothing.  (The paper has no counterpart: this
  * entry point exists for integration reasons only.)
  *

@@ -18,6 +18,7 @@ EXPORTED_SYMBOLS = (
     "flashd_attn_fwd", "flashd_attn_fwd_ex", "flashd_attn_fwd_f32", "flashd_attn_fwd_perkey",
     "flashd_splitk_workspace_bytes", "flashd_splitk_num_splits", "flashd_splitk_partial",
     "flashd_splitk_combine", "flashd_attn_fwd_splitk", "flashd_attn_fwd_splitk_static",
+    "flashd_gqa_num_splits", "flashd_gqa_partial", "flashd_attn_fwd_gqa",
     "flashd_attn_fwd_host", "flashd_skip_stats", "flashd_last_device_status", "flashd_status_string", "flashd_version", "flashd_launch_count",
 )
 
@@ -59,6 +60,9 @@ def lib() -> ctypes.CDLL:
             L.flashd_splitk_partial.argtypes = [vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_splitk_combine.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, vp]
             L.flashd_attn_fwd_splitk.argtypes = [vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
+            L.flashd_gqa_num_splits.argtypes = [ci, ci, ci, ci, ci]
+            L.flashd_gqa_partial.argtypes = [vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
+            L.flashd_attn_fwd_gqa.argtypes = [vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_attn_fwd_splitk_static.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_skip_stats.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, cf, cf, cf, cf, vp]
             L.flashd_attn_fwd_host.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp]
@@ -219,6 +223,51 @@ def flashd_attn_fwd_splitk(q, k, v, scale, num_splits=0, workspace=None, o=None,
     _check(lib().flashd_attn_fwd_splitk(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(workspace),
                                         workspace.numel() * workspace.element_size(), B, H, Nq, Nk, d,
                                         float(scale), int(num_splits), _stream_ptr(stream)), "flashd_attn_fwd_splitk")
+    return o
+
+
+MAX_GROUP = 8
+
+
+def _gqa_dims(q, k, v):
+    for t in (q, k, v):
+        if not (t.dim() == 4 and t.is_contiguous()):
+            raise ValueError("q, k, v must be contiguous [B, H, N, d] tensors")
+    B, Hq, Nq, d = q.shape
+    Bk, Hkv, Nk, dk = k.shape
+    if Nq != 1 or Bk != B or dk != d or tuple(v.shape) != tuple(k.shape) or Hkv == 0 or Hq % Hkv != 0:
+        raise ValueError(f"grouped-query shapes do not match: q {tuple(q.shape)} k {tuple(k.shape)} v {tuple(v.shape)}")
+    return B, Hkv, Hq // Hkv, Nk, d
+
+
+def flashd_gqa_num_splits(B, Hkv, G, Nk, d) -> int:
+    return int(lib().flashd_gqa_num_splits(B, Hkv, G, Nk, d))
+
+
+def flashd_gqa_partial(q, k, v, scale, num_splits, workspace=None, stream=None):
+    """Partial states ``[B,Hkv*G,1,num_splits,d+1]`` fp32 of the grouped-query split-K forward."""
+    import torch
+    B, Hkv, G, Nk, d = _gqa_dims(q, k, v)
+    if workspace is None:
+        workspace = torch.empty((B, Hkv * G, 1, num_splits, d + 1), dtype=torch.float32, device=q.device)
+    _check(lib().flashd_gqa_partial(_ptr(q), _ptr(k), _ptr(v), _ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), B, Hkv, G, Nk, d,
+                                    float(scale), int(num_splits), _stream_ptr(stream)), "flashd_gqa_partial")
+    return workspace
+
+
+def flashd_attn_fwd_gqa(q, k, v, scale, num_splits=0, workspace=None, o=None, stream=None):
+    """Grouped-query split-K forward: q ``[B,Hkv*G,1,d]``, k/v ``[B,Hkv,Nk,d]``."""
+    import torch
+    B, Hkv, G, Nk, d = _gqa_dims(q, k, v)
+    S = num_splits if num_splits > 0 else flashd_gqa_num_splits(B, Hkv, G, Nk, d)
+    if workspace is None:
+        workspace = torch.empty((B, Hkv * G, 1, max(S, 1), d + 1), dtype=torch.float32, device=q.device)
+    if o is None:
+        o = torch.empty_like(q)
+    _check(lib().flashd_attn_fwd_gqa(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), B, Hkv, G, Nk, d,
+                                     float(scale), int(num_splits), _stream_ptr(stream)), "flashd_attn_fwd_gqa")
     return o
 
 

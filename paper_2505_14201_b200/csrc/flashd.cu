@@ -14,6 +14,7 @@
 #include "flashd_decode.cuh"
 #include "flashd_perkey.cuh"
 #include "flashd_prefill.cuh"
+#include "flashd_gqa.cuh"
 #include "flashd_skipstats.cuh"
 
 namespace {
@@ -157,6 +158,31 @@ int launch_partial(const void* q, const void* k, const void* v, void* ws, long l
     splitk_partial_kernel<D><<<grid, C::kThreads, C::kSmemBytes, stream>>>(
         static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
         static_cast<const __nv_bfloat16*>(v), static_cast<float*>(ws), rows, Nq, Nk, scale * kLog2e, num_splits);
+    return after_launch();
+}
+
+template <int D>
+int launch_gqa_partial(const void* q, const void* k, const void* v, void* ws, int BHkv, int G, int Nk, float scale,
+                       int num_splits, cudaStream_t stream) {
+    using C = GqaCfg<D>;
+    CUtensorMap mk, mv;
+    if (!make_map(&mk, k, BHkv, Nk, D) || !make_map(&mv, v, BHkv, Nk, D)) return FLASHD_ERR_CUDA;
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FLASHD_ERR_CUDA;
+    if (!attr_set[dev]) {
+        if (cudaFuncSetAttribute(gqa_partial_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 C::kSmemBytes) != cudaSuccess)
+            return FLASHD_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    const int sms = sm_count();
+    if (sms <= 0) return FLASHD_ERR_CUDA;
+    const long long items = (long long)BHkv * num_splits;
+    const int grid = (int)(items < sms ? items : sms);
+    gqa_partial_kernel<D><<<grid, C::kThreads, C::kSmemBytes, stream>>>(
+        mk, mv, static_cast<const __nv_bfloat16*>(q), static_cast<float*>(ws), BHkv, G, Nk, scale * kLog2e,
+        num_splits);
     return after_launch();
 }
 
@@ -314,6 +340,35 @@ int flashd_attn_fwd_splitk(const void* q, const void* k, const void* v, void* o,
     int st = flashd_splitk_partial(q, k, v, workspace, workspace_bytes, B, H, Nq, Nk, d, scale, num_splits, stream);
     if (st != FLASHD_OK) return st;
     return flashd_splitk_combine(workspace, o, nullptr, B, H, Nq, d, num_splits, FLASHD_BF16, stream);
+}
+
+int flashd_gqa_num_splits(int B, int Hkv, int G, int Nk, int d) {
+    (void)G;
+    return flashd_splitk_num_splits(B, Hkv, 1, Nk, d);
+}
+
+int flashd_gqa_partial(const void* q, const void* k, const void* v, void* workspace, size_t workspace_bytes, int B,
+                       int Hkv, int G, int Nk, int d, float scale, int num_splits, void* stream) {
+    if (G < 1 || G > FLASHD_MAX_GROUP) return G < 1 ? FLASHD_ERR_SHAPE : FLASHD_ERR_UNSUPPORTED;
+    const int st = check_common(q, k, v, workspace, B, Hkv, 1, Nk, d, scale);
+    if (st != FLASHD_OK) return st;
+    if (d != 128 && d != 64) return FLASHD_ERR_UNSUPPORTED;
+    const int cs = check_splits(Nk, num_splits);
+    if (cs != FLASHD_OK) return cs;
+    if ((long long)B * Hkv * G > 0x7fffffffLL / FLASHD_MAX_SPLITS) return FLASHD_ERR_SHAPE;
+    if (workspace_bytes < flashd_splitk_workspace_bytes(B, Hkv * G, 1, d, num_splits)) return FLASHD_ERR_WORKSPACE;
+    const int BHkv = B * Hkv;
+    if (d == 128) return launch_gqa_partial<128>(q, k, v, workspace, BHkv, G, Nk, scale, num_splits, as_stream(stream));
+    return launch_gqa_partial<64>(q, k, v, workspace, BHkv, G, Nk, scale, num_splits, as_stream(stream));
+}
+
+int flashd_attn_fwd_gqa(const void* q, const void* k, const void* v, void* o, void* workspace, size_t workspace_bytes,
+                        int B, int Hkv, int G, int Nk, int d, float scale, int num_splits, void* stream) {
+    if (!o || !workspace) return FLASHD_ERR_NULL;
+    if (num_splits <= 0) num_splits = flashd_gqa_num_splits(B, Hkv, G, Nk, d);
+    const int st = flashd_gqa_partial(q, k, v, workspace, workspace_bytes, B, Hkv, G, Nk, d, scale, num_splits, stream);
+    if (st != FLASHD_OK) return st;
+    return flashd_splitk_combine(workspace, o, nullptr, B, Hkv * G, 1, d, num_splits, FLASHD_BF16, stream);
 }
 
 int flashd_attn_fwd_splitk_static(const void* q, const void* k, const void* v, void* o, int B, int H, int Nq,
