@@ -58,6 +58,11 @@ def _load():
             lib.oracle_split_merge.argtypes = [_D, _D, _D, _D, ci, ci, ci]
             lib.oracle_flashd_weights.argtypes = [_D, ci, _D, ci]
             lib.oracle_skip_stats.argtypes = [_D, _D, _LL, ci, ci, ci, ci, ci, cd, ci, _I, cd, cd, cd, cd, cd]
+            lib.oracle_attn_flashd_pwl.argtypes = [_D, _D, _D, _D, ci, ci, ci, ci, ci, cd, ci, _I,
+                                                   ci, _D, _D, ci, _D, _D, cd, cd, ci, cd, _LL]
+            lib.oracle_attn_flashd_pwl.restype = None
+            lib.oracle_pwl_eval.argtypes = [_D, _D, ci, cd]
+            lib.oracle_pwl_eval.restype = cd
             for f in ("oracle_attn_naive", "oracle_attn_alg1", "oracle_attn_alg2",
                       "oracle_attn_flashd", "oracle_attn_tiled", "oracle_split_merge",
                       "oracle_flashd_weights", "oracle_skip_stats"):
@@ -207,3 +212,29 @@ def skip_stats(q, k, scale, causal=False, q_index=None, lo=-6.0, hi=11.0, alo=-6
                               float(scale), int(bool(causal)), _pi(qi), float(lo), float(hi),
                               float(alo), float(ahi), float(near))
     return tuple(int(c) for c in counts)
+
+
+def pwl_eval(xs, ys, x) -> float:
+    """Continuous piece-wise linear function through the nodes (xs, ys), saturating outside."""
+    xs, ys = _f64(xs), _f64(ys)
+    return float(_load().oracle_pwl_eval(_p(xs), _p(ys), len(xs) - 1, float(x)))
+
+
+def attn_flashd_pwl(q, k, v, scale, causal=False, q_index=None, sig=None, ln=None, lo=-6.0, hi=11.0,
+                    range_mode=0, near=1e-4, return_counts=False):
+    """Sec. IV-B: Algorithm 3 with PWL sigmoid / ln.  ``sig`` and ``ln`` are (xs, ys) node
+    tables or None for the exact function; ``range_mode`` 0 saturates the sigmoid argument to
+    [lo, hi], 1 bypasses keys below lo and replaces the output above hi.  With
+    ``return_counts`` also returns (bypassed, replaced, near-threshold) step counts."""
+    q, k, v, B, H, Nq, Nk, d, qi = _prep(q, k, v, q_index)
+    o = np.empty((B, H, Nq, d))
+    sx, sy = (None, None) if sig is None else (_f64(sig[0]), _f64(sig[1]))
+    lx, ly = (None, None) if ln is None else (_f64(ln[0]), _f64(ln[1]))
+    counts = np.zeros(3, dtype=np.int64)
+    _load().oracle_attn_flashd_pwl(_p(q), _p(k), _p(v), _p(o), B, H, Nq, Nk, d, float(scale),
+                                   int(bool(causal)), _pi(qi),
+                                   0 if sx is None else len(sx) - 1, _p(sx), _p(sy),
+                                   0 if lx is None else len(lx) - 1, _p(lx), _p(ly),
+                                   float(lo), float(hi), int(range_mode), float(near),
+                                   counts.ctypes.data_as(_LL))
+    return (o, tuple(int(c) for c in counts)) if return_counts else o

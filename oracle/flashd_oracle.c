@@ -28,6 +28,8 @@
  *                       one score vector.
  *   oracle_skip_stats   Sec. III-C / Sec. V-B: how often s_i - s_{i-1} falls
  *                       outside [-6, 11].
+ *   oracle_attn_flashd_pwl  Sec. IV-B: Algorithm 3 with piece-wise linear
+ *                       sigmoid and ln and a confined sigmoid input range.
  *
  * Masking is not in the paper (it treats one query over N keys).  Reading
  * taken here: a key that a query may not see is removed from that query's key
@@ -39,6 +41,11 @@
  * example, closed forms, invariants).  oracle_skip_stats: parity unpinned
  * against the paper's Table I (needs model weights and datasets that are not
  * available); it is pinned only by brute-force counting on small inputs.
+ * oracle_attn_flashd_pwl: parity unpinned against the paper (its PWL
+ * coefficients are not printed and it reports no accuracy figure); it is
+ * pinned by its limits: exact functions and an unbounded range give
+ * oracle_attn_flashd, a bypassed key gives the recurrence without that key,
+ * and refined tables converge at second order.
  */
 #include <math.h>
 #include <stdlib.h>
@@ -435,4 +442,80 @@ void oracle_skip_stats(const double* q, const double* k, long long* counts,
     }
     counts[0] = total; counts[1] = below; counts[2] = above;
     counts[3] = abelow; counts[4] = aabove; counts[5] = nnear;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Sec. IV-B: Algorithm 3 with the sigmoid and the natural logarithm replaced
+ * by continuous piece-wise linear (PWL) approximations, and the sigmoid input
+ * confined to a range [lo, hi] (the paper: 8 segments each, range [-6, 11]).
+ *
+ * A PWL function is given by n_seg + 1 nodes (x_0 < ... < x_n, y_0 .. y_n):
+ * linear between neighbouring nodes, equal to the end value outside [x_0, x_n]
+ * ("no computation is required outside this range").  The paper does not print
+ * its coefficients, so the tables are inputs here.  n_seg = 0 selects the exact
+ * function instead (sigma, resp. ln; with both exact, ln w is taken as
+ * ln sigma(x), so that lo = -inf, hi = +inf reproduces oracle_attn_flashd).   */
+double oracle_pwl_eval(const double* xs, const double* ys, int n_seg, double x) {
+    if (x <= xs[0]) return ys[0];
+    if (x >= xs[n_seg]) return ys[n_seg];
+    int m = 0;
+    while (m + 1 < n_seg && x >= xs[m + 1]) ++m;          /* segment with xs[m] <= x < xs[m+1] */
+    return ys[m] + (x - xs[m]) * (ys[m + 1] - ys[m]) / (xs[m + 1] - xs[m]);
+}
+
+/* The carried state is the paper's (s_{i-1}, ln w_{i-1}, o_{i-1}).  Per key,
+ * with x = s_i - s_{i-1} + ln w_{i-1} (argument of Eq. (w-last)):
+ *   range_mode 0 (saturate): x is clamped to [lo, hi]; w = SIG(x); ln w = LN(w).
+ *   range_mode 1 (bypass, Sec. III-C read on x): x < lo: the key is bypassed -
+ *       no output update and the state stays as it was, which is the recurrence
+ *       over the key sequence with that key removed; x > hi: w = 1, the output
+ *       is replaced by v_i (the recurrence restarted at key i); otherwise as in
+ *       mode 0.
+ * counts (nullable, [3]) receives the number of bypassed keys, of replacements,
+ * and of steps whose x lies within `near` of lo or hi (where the fp32 device
+ * code may decide differently).                                              */
+void oracle_attn_flashd_pwl(const double* q, const double* k, const double* v, double* o,
+                            int B, int H, int Nq, int Nk, int d,
+                            double scale, int causal, const int* q_index,
+                            int sig_n, const double* sig_x, const double* sig_y,
+                            int ln_n, const double* ln_x, const double* ln_y,
+                            double lo, double hi, int range_mode, double near,
+                            long long* counts) {
+    long long n_skip = 0, n_repl = 0, n_near = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1) reduction(+ : n_skip, n_repl, n_near)
+    for (int bh = 0; bh < B * H; ++bh) {
+        for (int i = 0; i < Nq; ++i) {
+            const double* qi = q + ((size_t)bh * Nq + i) * d;
+            const double* kb = k + (size_t)bh * Nk * d;
+            const double* vb = v + (size_t)bh * Nk * d;
+            double* oi = o + ((size_t)bh * Nq + i) * d;
+            int nv = n_visible(q_global(q_index, i), Nk, causal);
+            double s_prev = 0.0, lnw = 0.0;
+            for (int c = 0; c < d; ++c) oi[c] = (nv > 0) ? 0.0 : NAN;
+            for (int j = 0; j < nv; ++j) {
+                double s = dot_scaled(qi, kb + (size_t)j * d, d, scale);
+                const double* vj = vb + (size_t)j * d;
+                double w;
+                if (j == 0) {
+                    w = 1.0; lnw = 0.0;
+                } else {
+                    double x = s - s_prev + lnw;
+                    if (fabs(x - lo) < near || fabs(x - hi) < near) ++n_near;
+                    if (range_mode == 1 && x < lo) { ++n_skip; continue; }
+                    if (range_mode == 1 && x > hi) {
+                        ++n_repl; w = 1.0; lnw = 0.0;
+                    } else {
+                        if (x < lo) x = lo;
+                        if (x > hi) x = hi;
+                        w = sig_n > 0 ? oracle_pwl_eval(sig_x, sig_y, sig_n, x) : sigmoid(x);
+                        if (ln_n > 0) lnw = oracle_pwl_eval(ln_x, ln_y, ln_n, w);
+                        else lnw = sig_n > 0 ? log(w) : log_sigmoid(x);
+                    }
+                }
+                for (int c = 0; c < d; ++c) oi[c] = oi[c] + (vj[c] - oi[c]) * w;
+                s_prev = s;
+            }
+        }
+    }
+    if (counts) { counts[0] = n_skip; counts[1] = n_repl; counts[2] = n_near; }
 }

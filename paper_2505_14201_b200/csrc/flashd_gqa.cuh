@@ -43,7 +43,7 @@ struct GqaCfg {
     static constexpr int kSmemBytes = kStages * kStageBytes + kMergeFloats * 4 + 256 + 1024;
 };
 
-enum { kWaitGqaFull = 0x200, kWaitGqaEmpty = 0x201, kWaitGqaMergeReady = 0x202, kWaitGqaMergeFree = 0x203 };
+enum { kWaitGqaFull = 0x300, kWaitGqaEmpty = 0x301, kWaitGqaMergeReady = 0x302, kWaitGqaMergeFree = 0x303 };
 
 // Four 8x8 b16 matrices from shared memory; lane l supplies the address of row
 // l%8 of matrix l/8.  Plain form: thread t receives elements (row t/4, columns
@@ -63,13 +63,11 @@ __device__ __forceinline__ void ldsm_x4_trans(uint32_t saddr, uint32_t (&r)[4]) 
 // Only rows 0..7 of A are populated (a1 = a3 = 0), so only d0, d1 carry results;
 // the accumulators of rows 8..15 are fed zeros and dropped.
 __device__ __forceinline__ void mma_rows8(float& d0, float& d1, uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
-    float x2, x3;
+    [[maybe_unused]] float x2, x3;
     asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
         "{%0, %1, %10, %10};"
         : "+f"(d0), "+f"(d1), "=f"(x2), "=f"(x3)
         : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.f));
-    (void)x2;
-    (void)x3;
 }
 
 template <int D>

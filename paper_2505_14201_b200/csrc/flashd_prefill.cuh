@@ -159,6 +159,8 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
           "r"(taddr)
         : "memory");
 }
+// setmaxnreg is a warpgroup instruction: the four warps of a warpgroup (0-3, 4-7, 8-11, 12-15)
+// must all execute it with the same value, or they wait for each other forever.
 template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
