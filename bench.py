@@ -358,6 +358,48 @@ def run_skip_stats(fd, synth, torch, device):
                       "data": "synthetic", "workloads": out}), flush=True)
 
 
+def run_pwl_study(fd, synth, torch, device):
+    """Sec. IV-B in numbers: output error of Algorithm 3 when the sigmoid and ln are 8-segment PWL
+    fits and the sigmoid argument is confined to [-6, 11], against the exact per-key kernel, on the
+    synthetic workloads (config 4 on its first 4 batch elements)."""
+    import dataclasses
+    from paper_2505_14201_b200 import pwl
+    sig, ln = pwl.paper_tables()
+    variants = {"exact_saturate": (None, None, 0), "exact_bypass": (None, None, 1),
+                "pwl8_saturate": (sig, ln, 0), "pwl8_bypass": (sig, ln, 1)}
+    out = {}
+    for name in ("c0", "c1", "c2", "c3", "c4"):
+        w = synth.WORKLOADS[name]
+        if name == "c4":
+            w = dataclasses.replace(w, B=4)
+        q, k, v = synth.make_inputs(w, device=device)
+        sc = f32(w.scale)
+        ref = fd.flashd_attn_fwd_perkey(q, k, v, sc, w.causal, out_dtype=torch.float32)
+        steps = (w.B * w.H * (w.Nq * (w.Nq + 1) // 2 if w.causal else w.Nq * w.Nk))
+        res = {}
+        for vn, (st, lt, mode) in variants.items():
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record()
+            got, cnt = fd.flashd_attn_fwd_pwl(q, k, v, sc, w.causal, sig=st, ln=lt, lo=-6.0, hi=11.0, range_mode=mode,
+                                              out_dtype=torch.float32, return_counts=True)
+            e1.record(); torch.cuda.synchronize()
+            err = (got - ref).abs()
+            res[vn] = {"max_abs_err": float(err.max()), "mean_abs_err": float(err.mean()),
+                       "bypassed_pct": 100.0 * cnt[0] / steps, "replaced_pct": 100.0 * cnt[1] / steps,
+                       "ms": e0.elapsed_time(e1)}
+            del got, err
+        out[name] = res
+        del q, k, v, ref
+        torch.cuda.empty_cache()
+    st_, detail = fd.flashd_last_device_status()
+    if st_ != 0:
+        raise SystemExit(f"device status {st_} {detail}")
+    print(json.dumps({"metric": "pwl_output_error_vs_exact", "segments": 8, "range": [-6, 11], "data": "synthetic",
+                      "sigmoid_table_max_err": pwl.max_error(sig, pwl.sigmoid, *pwl.SIGMOID_RANGE),
+                      "ln_table_max_err": pwl.max_error(ln, __import__("numpy").log, *pwl.ln_range()),
+                      "workloads": out}), flush=True)
+
+
 def run_gqa(fd, synth, torch, device, peaks, steps):
     """Grouped-query decode: config 4 with its 32 query heads sharing 32/G K/V heads.  The K/V
     stream (the algorithmic bytes) shrinks by G, the arithmetic per K/V byte grows by G."""
@@ -400,6 +442,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--skip-stats", action="store_true",
                     help="print the bypassable-update statistic (Sec. III-C / V-B) of every workload instead of timing")
+    ap.add_argument("--pwl-study", action="store_true",
+                    help="print the output error of the PWL / confined-range datapath model (Sec. IV-B) instead of timing")
     ap.add_argument("--gqa", action="store_true",
                     help="time the grouped-query decode variant (config 4 with shared K/V heads) instead")
     ap.add_argument("--batch", type=int, default=0,
@@ -435,6 +479,9 @@ def main():
         run_skip_stats(fd, synth, torch, device)
         return
 
+    if args.pwl_study:
+        run_pwl_study(fd, synth, torch, device)
+        return
     if args.gqa:
         run_gqa(fd, synth, torch, device, peaks, min(args.steps, 30))
         return

@@ -104,6 +104,38 @@ int flashd_attn_fwd_perkey(const void* q, const void* k, const void* v, void* o,
                            void* stream);
 
 /* ------------------------------------------------------------------------
+ * Algorithm 3 with piece-wise linear sigmoid and ln (Sec. IV-B): the numerical
+ * model of the paper's datapath, for accuracy studies.  One key at a time like
+ * flashd_attn_fwd_perkey; not a throughput path.
+ *
+ * A table describes a continuous piece-wise linear function by n + 1 nodes:
+ * x[0] < ... < x[n] with values y[0..n]; linear in between, y[0] / y[n]
+ * outside.  sig_* replaces the sigmoid of Eq. (w-last), ln_* replaces the
+ * natural logarithm that yields ln w_i from w_i.  n = 0 (pointers may be NULL)
+ * selects the exact function.  1 <= n <= FLASHD_PWL_MAX_SEGMENTS otherwise.
+ * The tables are HOST arrays of n + 1 floats, read during the call (the caller
+ * may free them on return).  The paper uses n = 8 for both and does not print
+ * its coefficients.
+ *
+ * The sigmoid argument x = s_i - s_(i-1) + ln w_(i-1) is confined to [lo, hi]
+ * (the paper: [-6, 11]; -INFINITY / +INFINITY lift a bound):
+ *   range_mode 0: x is clamped to the range;
+ *   range_mode 1: x < lo bypasses the key - no output update, carried state
+ *                 unchanged (Sec. III-C); x > hi replaces the output by v_i
+ *                 (w_i = 1).
+ * counts: nullable DEVICE pointer to two 64-bit counters, incremented by the
+ * number of bypassed keys and of replacements (the caller zeroes them).
+ * in_dtype / out_dtype, d, layout and errors as flashd_attn_fwd_perkey;
+ * a malformed table or range returns FLASHD_ERR_SHAPE.                       */
+#define FLASHD_PWL_MAX_SEGMENTS 64
+int flashd_attn_fwd_pwl(const void* q, const void* k, const void* v, void* o,
+                        unsigned long long* counts, int in_dtype, int out_dtype,
+                        int B, int H, int Nq, int Nk, int d, float scale, int causal,
+                        int sig_n, const float* sig_x, const float* sig_y,
+                        int ln_n, const float* ln_x, const float* ln_y,
+                        float lo, float hi, int range_mode, void* stream);
+
+/* ------------------------------------------------------------------------
  * Split-K forward for long key sequences and few queries (decode).
  * Non-causal, bf16 in, d = 128 or 64.
  *

@@ -18,7 +18,7 @@ EXPORTED_SYMBOLS = (
     "flashd_attn_fwd", "flashd_attn_fwd_ex", "flashd_attn_fwd_f32", "flashd_attn_fwd_perkey",
     "flashd_splitk_workspace_bytes", "flashd_splitk_num_splits", "flashd_splitk_partial",
     "flashd_splitk_combine", "flashd_attn_fwd_splitk", "flashd_attn_fwd_splitk_static",
-    "flashd_gqa_num_splits", "flashd_gqa_partial", "flashd_attn_fwd_gqa",
+    "flashd_gqa_num_splits", "flashd_gqa_partial", "flashd_attn_fwd_gqa", "flashd_attn_fwd_pwl",
     "flashd_attn_fwd_host", "flashd_skip_stats", "flashd_last_device_status", "flashd_status_string", "flashd_version", "flashd_launch_count",
 )
 
@@ -60,6 +60,9 @@ def lib() -> ctypes.CDLL:
             L.flashd_splitk_partial.argtypes = [vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_splitk_combine.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, vp]
             L.flashd_attn_fwd_splitk.argtypes = [vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
+            fp = ctypes.POINTER(ctypes.c_float)
+            L.flashd_attn_fwd_pwl.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, ci,
+                                              ci, fp, fp, ci, fp, fp, cf, cf, ci, vp]
             L.flashd_gqa_num_splits.argtypes = [ci, ci, ci, ci, ci]
             L.flashd_gqa_partial.argtypes = [vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_attn_fwd_gqa.argtypes = [vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
@@ -177,6 +180,42 @@ def flashd_attn_fwd_perkey(q, k, v, scale, causal=False, out_dtype=None, return_
                                         _dtype_code(o), B, H, Nq, Nk, d, float(scale), int(bool(causal)),
                                         _stream_ptr(stream)), "flashd_attn_fwd_perkey")
     return (o, lse) if return_lse else o
+
+
+PWL_MAX_SEGMENTS = 64
+
+
+def _host_table(tab):
+    """(xs, ys) -> (n, float* x, float* y, keep-alive); None -> exact function."""
+    if tab is None:
+        return 0, None, None, None
+    xs = [float(t) for t in tab[0]]
+    ys = [float(t) for t in tab[1]]
+    if len(xs) != len(ys) or len(xs) < 2:
+        raise ValueError("a PWL table needs matching node lists of at least two nodes")
+    ax = (ctypes.c_float * len(xs))(*xs)
+    ay = (ctypes.c_float * len(ys))(*ys)
+    return len(xs) - 1, ax, ay, (ax, ay)
+
+
+def flashd_attn_fwd_pwl(q, k, v, scale, causal=False, sig=None, ln=None, lo=-6.0, hi=11.0, range_mode=0,
+                        out_dtype=None, return_counts=False, o=None, stream=None):
+    """Algorithm 3 with piece-wise linear sigmoid / ln tables (Sec. IV-B accuracy model).
+    ``sig`` / ``ln``: (xs, ys) node lists or None for the exact function."""
+    import torch
+    B, H, Nq, Nk, d = _dims(q, k, v)
+    out_dtype = q.dtype if out_dtype is None else out_dtype
+    if o is None:
+        o = torch.empty(q.shape, dtype=out_dtype, device=q.device)
+    counts = torch.zeros(2, dtype=torch.int64, device=q.device) if return_counts else None
+    sn, sx, sy, keep1 = _host_table(sig)
+    ln_n, lx, ly, keep2 = _host_table(ln)
+    _check(lib().flashd_attn_fwd_pwl(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(counts), _dtype_code(q),
+                                     _dtype_code(o), B, H, Nq, Nk, d, float(scale), int(bool(causal)),
+                                     sn, sx, sy, ln_n, lx, ly, float(lo), float(hi), int(range_mode),
+                                     _stream_ptr(stream)), "flashd_attn_fwd_pwl")
+    del keep1, keep2
+    return (o, tuple(int(c) for c in counts.cpu())) if return_counts else o
 
 
 def flashd_splitk_workspace_bytes(B, H, Nq, d, num_splits) -> int:

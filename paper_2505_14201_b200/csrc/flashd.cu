@@ -15,6 +15,7 @@
 #include "flashd_perkey.cuh"
 #include "flashd_prefill.cuh"
 #include "flashd_gqa.cuh"
+#include "flashd_pwl.cuh"
 #include "flashd_skipstats.cuh"
 
 namespace {
@@ -136,6 +137,44 @@ int launch_perkey_t(const void* q, const void* k, const void* v, void* o, float*
         default: return FLASHD_ERR_UNSUPPORTED;
     }
     return after_launch();
+}
+
+template <typename TIn, typename TOut>
+int launch_pwl_t(const void* q, const void* k, const void* v, void* o, unsigned long long* counts, long long rows,
+                 int Nq, int Nk, int d, float scale, int causal, const PwlTables& tab, float lo, float hi,
+                 int range_mode, cudaStream_t stream) {
+    const int warps = 4;
+    const long long blocks = (rows + warps - 1) / warps;
+    if (blocks > 0x7fffffffLL) return FLASHD_ERR_SHAPE;
+    const TIn* qq = static_cast<const TIn*>(q);
+    const TIn* kk = static_cast<const TIn*>(k);
+    const TIn* vv = static_cast<const TIn*>(v);
+    TOut* oo = static_cast<TOut*>(o);
+    const unsigned g = (unsigned)blocks;
+    switch (d) {
+        case 32: perkey_pwl_kernel<TIn, TOut, 1><<<g, warps * 32, 0, stream>>>(qq, kk, vv, oo, counts, rows, Nq, Nk, scale, causal, tab, lo, hi, range_mode); break;
+        case 64: perkey_pwl_kernel<TIn, TOut, 2><<<g, warps * 32, 0, stream>>>(qq, kk, vv, oo, counts, rows, Nq, Nk, scale, causal, tab, lo, hi, range_mode); break;
+        case 128: perkey_pwl_kernel<TIn, TOut, 4><<<g, warps * 32, 0, stream>>>(qq, kk, vv, oo, counts, rows, Nq, Nk, scale, causal, tab, lo, hi, range_mode); break;
+        case 256: perkey_pwl_kernel<TIn, TOut, 8><<<g, warps * 32, 0, stream>>>(qq, kk, vv, oo, counts, rows, Nq, Nk, scale, causal, tab, lo, hi, range_mode); break;
+        default: return FLASHD_ERR_UNSUPPORTED;
+    }
+    return after_launch();
+}
+
+// copies one host table into the kernel-parameter block; false if malformed
+bool fill_table(int n, const float* x, const float* y, int* n_out, float* xs, float* ys) {
+    for (int t = 0; t <= FLASHD_PWL_MAX_SEGMENTS; ++t) { xs[t] = 0.f; ys[t] = 0.f; }
+    *n_out = 0;
+    if (n == 0) return true;
+    if (n < 0 || n > FLASHD_PWL_MAX_SEGMENTS || !x || !y) return false;
+    for (int t = 0; t <= n; ++t) {
+        if (!std::isfinite(x[t]) || !std::isfinite(y[t])) return false;
+        if (t > 0 && !(x[t] > x[t - 1])) return false;
+        xs[t] = x[t];
+        ys[t] = y[t];
+    }
+    *n_out = n;
+    return true;
 }
 
 template <int D>
@@ -270,6 +309,29 @@ int flashd_attn_fwd_perkey(const void* q, const void* k, const void* v, void* o,
         return launch_perkey_t<__nv_bfloat16, __nv_bfloat16>(q, k, v, o, lse_out, rows, Nq, Nk, d, scale, causal, s);
     if (in_dtype == FLASHD_BF16 && out_dtype == FLASHD_F32)
         return launch_perkey_t<__nv_bfloat16, float>(q, k, v, o, lse_out, rows, Nq, Nk, d, scale, causal, s);
+    return FLASHD_ERR_UNSUPPORTED;
+}
+
+int flashd_attn_fwd_pwl(const void* q, const void* k, const void* v, void* o, unsigned long long* counts,
+                        int in_dtype, int out_dtype, int B, int H, int Nq, int Nk, int d, float scale, int causal,
+                        int sig_n, const float* sig_x, const float* sig_y, int ln_n, const float* ln_x,
+                        const float* ln_y, float lo, float hi, int range_mode, void* stream) {
+    const int st = check_common(q, k, v, o, B, H, Nq, Nk, d, scale);
+    if (st != FLASHD_OK) return st;
+    if (d != 32 && d != 64 && d != 128 && d != 256) return FLASHD_ERR_UNSUPPORTED;
+    if (range_mode != 0 && range_mode != 1) return FLASHD_ERR_SHAPE;
+    if (std::isnan(lo) || std::isnan(hi) || !(lo <= hi)) return FLASHD_ERR_SHAPE;
+    PwlTables tab;
+    if (!fill_table(sig_n, sig_x, sig_y, &tab.sig_n, tab.sig_x, tab.sig_y)) return FLASHD_ERR_SHAPE;
+    if (!fill_table(ln_n, ln_x, ln_y, &tab.ln_n, tab.ln_x, tab.ln_y)) return FLASHD_ERR_SHAPE;
+    const long long rows = (long long)B * H * Nq;
+    cudaStream_t s = as_stream(stream);
+    if (in_dtype == FLASHD_F32 && out_dtype == FLASHD_F32)
+        return launch_pwl_t<float, float>(q, k, v, o, counts, rows, Nq, Nk, d, scale, causal, tab, lo, hi, range_mode, s);
+    if (in_dtype == FLASHD_BF16 && out_dtype == FLASHD_BF16)
+        return launch_pwl_t<__nv_bfloat16, __nv_bfloat16>(q, k, v, o, counts, rows, Nq, Nk, d, scale, causal, tab, lo, hi, range_mode, s);
+    if (in_dtype == FLASHD_BF16 && out_dtype == FLASHD_F32)
+        return launch_pwl_t<__nv_bfloat16, float>(q, k, v, o, counts, rows, Nq, Nk, d, scale, causal, tab, lo, hi, range_mode, s);
     return FLASHD_ERR_UNSUPPORTED;
 }
 
