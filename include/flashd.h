@@ -94,7 +94,8 @@ int flashd_attn_fwd_ex(const void* q, const void* k, const void* v, void* o, flo
  *
  * flashd_attn_fwd_f32: fp32 in, fp32 out.
  * flashd_attn_fwd_perkey: in_dtype / out_dtype in {FLASHD_BF16, FLASHD_F32}.
- * d must be 32, 64, 128 or 256.  lse_out nullable.                        */
+ * d must be 16, 32, 64, 128 or 256 (the hidden sizes of the paper's evaluation,
+ * Sec. V-A).  lse_out nullable.                        */
 int flashd_attn_fwd_f32(const void* q, const void* k, const void* v, void* o,
                         int B, int H, int Nq, int Nk, int d, float scale, int causal,
                         void* stream);

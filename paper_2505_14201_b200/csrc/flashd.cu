@@ -130,10 +130,11 @@ int launch_perkey_t(const void* q, const void* k, const void* v, void* o, float*
     const TIn* vv = static_cast<const TIn*>(v);
     TOut* oo = static_cast<TOut*>(o);
     switch (d) {
-        case 32: perkey_kernel<TIn, TOut, 1><<<(unsigned)blocks, warps * 32, 0, stream>>>(qq, kk, vv, oo, lse, rows, Nq, Nk, scale, causal); break;
-        case 64: perkey_kernel<TIn, TOut, 2><<<(unsigned)blocks, warps * 32, 0, stream>>>(qq, kk, vv, oo, lse, rows, Nq, Nk, scale, causal); break;
-        case 128: perkey_kernel<TIn, TOut, 4><<<(unsigned)blocks, warps * 32, 0, stream>>>(qq, kk, vv, oo, lse, rows, Nq, Nk, scale, causal); break;
-        case 256: perkey_kernel<TIn, TOut, 8><<<(unsigned)blocks, warps * 32, 0, stream>>>(qq, kk, vv, oo, lse, rows, Nq, Nk, scale, causal); break;
+        case 16:
+        case 32: perkey_kernel<TIn, TOut, 1><<<(unsigned)blocks, warps * 32, 0, stream>>>(qq, kk, vv, oo, lse, rows, Nq, Nk, scale, causal, d); break;
+        case 64: perkey_kernel<TIn, TOut, 2><<<(unsigned)blocks, warps * 32, 0, stream>>>(qq, kk, vv, oo, lse, rows, Nq, Nk, scale, causal, d); break;
+        case 128: perkey_kernel<TIn, TOut, 4><<<(unsigned)blocks, warps * 32, 0, stream>>>(qq, kk, vv, oo, lse, rows, Nq, Nk, scale, causal, d); break;
+        case 256: perkey_kernel<TIn, TOut, 8><<<(unsigned)blocks, warps * 32, 0, stream>>>(qq, kk, vv, oo, lse, rows, Nq, Nk, scale, causal, d); break;
         default: return FLASHD_ERR_UNSUPPORTED;
     }
     return after_launch();
@@ -152,10 +153,11 @@ int launch_pwl_t(const void* q, const void* k, const void* v, void* o, unsigned 
     TOut* oo = static_cast<TOut*>(o);
     const unsigned g = (unsigned)blocks;
     switch (d) {
-        case 32: perkey_pwl_kernel<TIn, TOut, 1><<<g, warps * 32, 0, stream>>>(qq, kk, vv, oo, counts, rows, Nq, Nk, scale, causal, tab, lo, hi, range_mode); break;
-        case 64: perkey_pwl_kernel<TIn, TOut, 2><<<g, warps * 32, 0, stream>>>(qq, kk, vv, oo, counts, rows, Nq, Nk, scale, causal, tab, lo, hi, range_mode); break;
-        case 128: perkey_pwl_kernel<TIn, TOut, 4><<<g, warps * 32, 0, stream>>>(qq, kk, vv, oo, counts, rows, Nq, Nk, scale, causal, tab, lo, hi, range_mode); break;
-        case 256: perkey_pwl_kernel<TIn, TOut, 8><<<g, warps * 32, 0, stream>>>(qq, kk, vv, oo, counts, rows, Nq, Nk, scale, causal, tab, lo, hi, range_mode); break;
+        case 16:
+        case 32: perkey_pwl_kernel<TIn, TOut, 1><<<g, warps * 32, 0, stream>>>(qq, kk, vv, oo, counts, rows, Nq, Nk, scale, causal, tab, lo, hi, range_mode, d); break;
+        case 64: perkey_pwl_kernel<TIn, TOut, 2><<<g, warps * 32, 0, stream>>>(qq, kk, vv, oo, counts, rows, Nq, Nk, scale, causal, tab, lo, hi, range_mode, d); break;
+        case 128: perkey_pwl_kernel<TIn, TOut, 4><<<g, warps * 32, 0, stream>>>(qq, kk, vv, oo, counts, rows, Nq, Nk, scale, causal, tab, lo, hi, range_mode, d); break;
+        case 256: perkey_pwl_kernel<TIn, TOut, 8><<<g, warps * 32, 0, stream>>>(qq, kk, vv, oo, counts, rows, Nq, Nk, scale, causal, tab, lo, hi, range_mode, d); break;
         default: return FLASHD_ERR_UNSUPPORTED;
     }
     return after_launch();
@@ -300,7 +302,7 @@ int flashd_attn_fwd_perkey(const void* q, const void* k, const void* v, void* o,
                            void* stream) {
     const int st = check_common(q, k, v, o, B, H, Nq, Nk, d, scale);
     if (st != FLASHD_OK) return st;
-    if (d != 32 && d != 64 && d != 128 && d != 256) return FLASHD_ERR_UNSUPPORTED;
+    if (d != 16 && d != 32 && d != 64 && d != 128 && d != 256) return FLASHD_ERR_UNSUPPORTED;
     const long long rows = (long long)B * H * Nq;
     cudaStream_t s = as_stream(stream);
     if (in_dtype == FLASHD_F32 && out_dtype == FLASHD_F32)
@@ -318,7 +320,7 @@ int flashd_attn_fwd_pwl(const void* q, const void* k, const void* v, void* o, un
                         const float* ln_y, float lo, float hi, int range_mode, void* stream) {
     const int st = check_common(q, k, v, o, B, H, Nq, Nk, d, scale);
     if (st != FLASHD_OK) return st;
-    if (d != 32 && d != 64 && d != 128 && d != 256) return FLASHD_ERR_UNSUPPORTED;
+    if (d != 16 && d != 32 && d != 64 && d != 128 && d != 256) return FLASHD_ERR_UNSUPPORTED;
     if (range_mode != 0 && range_mode != 1) return FLASHD_ERR_SHAPE;
     if (std::isnan(lo) || std::isnan(hi) || !(lo <= hi)) return FLASHD_ERR_SHAPE;
     PwlTables tab;
@@ -464,7 +466,7 @@ int flashd_skip_stats(const void* q, const void* k, unsigned long long* counts, 
     if (B <= 0 || H <= 0 || Nq <= 0 || Nk <= 0 || d <= 0 || !std::isfinite(scale)) return FLASHD_ERR_SHAPE;
     if (!(lo <= hi) || !(alo <= ahi)) return FLASHD_ERR_SHAPE;
     if (!aligned16(q) || !aligned16(k) || (reinterpret_cast<uintptr_t>(counts) & 7u)) return FLASHD_ERR_ALIGN;
-    if (d != 32 && d != 64 && d != 128 && d != 256) return FLASHD_ERR_UNSUPPORTED;
+    if (d != 16 && d != 32 && d != 64 && d != 128 && d != 256) return FLASHD_ERR_UNSUPPORTED;
     if (in_dtype != FLASHD_BF16 && in_dtype != FLASHD_F32) return FLASHD_ERR_UNSUPPORTED;
     const long long rows = (long long)B * H * Nq;
     const int warps = 4;

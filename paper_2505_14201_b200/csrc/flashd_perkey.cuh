@@ -23,8 +23,8 @@ template <typename TIn, typename TOut, int E>
 __global__ void __launch_bounds__(128)
 perkey_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* __restrict__ v,
               TOut* __restrict__ o, float* __restrict__ lse, long long rows, int Nq, int Nk,
-              float scale, int causal) {
-    constexpr int D = 32 * E;
+              float scale, int causal, int D) {
+    // D = row length: 32*E, or 16 with E = 1 (lanes 16..31 then hold no column)
     const int lane = threadIdx.x & 31;
     const long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (row >= rows) return;
@@ -32,11 +32,12 @@ perkey_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* _
     const int i = (int)(row - bh * Nq);
     const int nv = causal ? min(i + 1, Nk) : Nk;
 
+    const bool active = lane * E < D;
     double qd[E];
     float of[E];
     const TIn* qrow = q + row * D + lane * E;
 #pragma unroll
-    for (int e = 0; e < E; ++e) { qd[e] = (double)to_f32<TIn>(qrow[e]); of[e] = 0.f; }
+    for (int e = 0; e < E; ++e) { qd[e] = active ? (double)to_f32<TIn>(qrow[e]) : 0.0; of[e] = 0.f; }
 
     const TIn* kb = k + bh * (long long)Nk * D + lane * E;
     const TIn* vb = v + bh * (long long)Nk * D + lane * E;
@@ -47,8 +48,8 @@ perkey_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* _
         float kf[E], vf[E];
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-            kf[e] = to_f32<TIn>(kb[(long long)j * D + e]);
-            vf[e] = to_f32<TIn>(vb[(long long)j * D + e]);
+            kf[e] = active ? to_f32<TIn>(kb[(long long)j * D + e]) : 0.f;
+            vf[e] = active ? to_f32<TIn>(vb[(long long)j * D + e]) : 0.f;
         }
         double part = 0.0;
 #pragma unroll
@@ -80,7 +81,8 @@ perkey_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* _
 
     TOut* orow = o + row * D + lane * E;
 #pragma unroll
-    for (int e = 0; e < E; ++e) orow[e] = from_f32<TOut>(of[e]);
+    for (int e = 0; e < E; ++e)
+        if (active) orow[e] = from_f32<TOut>(of[e]);
     if (lse != nullptr && lane == 0) lse[row] = (float)(s_prev - lnw);
 }
 

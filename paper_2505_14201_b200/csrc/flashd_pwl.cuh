@@ -35,8 +35,8 @@ __global__ void __launch_bounds__(128)
 perkey_pwl_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* __restrict__ v,
                   TOut* __restrict__ o, unsigned long long* __restrict__ counts, long long rows, int Nq, int Nk,
                   float scale, int causal, const __grid_constant__ PwlTables tab, float lo, float hi,
-                  int range_mode) {
-    constexpr int D = 32 * E;
+                  int range_mode, int D) {
+    // D = row length: 32*E, or 16 with E = 1 (lanes 16..31 then hold no column)
     __shared__ float sx[FLASHD_PWL_MAX_SEGMENTS + 1], sy[FLASHD_PWL_MAX_SEGMENTS + 1];
     __shared__ float lx[FLASHD_PWL_MAX_SEGMENTS + 1], ly[FLASHD_PWL_MAX_SEGMENTS + 1];
     for (int t = threadIdx.x; t <= FLASHD_PWL_MAX_SEGMENTS; t += blockDim.x) {
@@ -50,11 +50,12 @@ perkey_pwl_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TI
     const int i = (int)(row - bh * Nq);
     const int nv = causal ? min(i + 1, Nk) : Nk;
 
+    const bool active = lane * E < D;
     double qd[E];
     float of[E];
     const TIn* qrow = q + row * D + lane * E;
 #pragma unroll
-    for (int e = 0; e < E; ++e) { qd[e] = (double)to_f32<TIn>(qrow[e]); of[e] = 0.f; }
+    for (int e = 0; e < E; ++e) { qd[e] = active ? (double)to_f32<TIn>(qrow[e]) : 0.0; of[e] = 0.f; }
     const TIn* kb = k + bh * (long long)Nk * D + lane * E;
     const TIn* vb = v + bh * (long long)Nk * D + lane * E;
     const double scale_d = (double)scale;
@@ -65,8 +66,8 @@ perkey_pwl_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TI
         float kf[E], vf[E];
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-            kf[e] = to_f32<TIn>(kb[(long long)j * D + e]);
-            vf[e] = to_f32<TIn>(vb[(long long)j * D + e]);
+            kf[e] = active ? to_f32<TIn>(kb[(long long)j * D + e]) : 0.f;
+            vf[e] = active ? to_f32<TIn>(vb[(long long)j * D + e]) : 0.f;
         }
         double part = 0.0;
 #pragma unroll
@@ -108,7 +109,8 @@ perkey_pwl_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TI
 
     TOut* orow = o + row * D + lane * E;
 #pragma unroll
-    for (int e = 0; e < E; ++e) orow[e] = from_f32<TOut>(of[e]);
+    for (int e = 0; e < E; ++e)
+        if (active) orow[e] = from_f32<TOut>(of[e]);
     if (counts != nullptr && lane == 0) {
         if (n_skip) atomicAdd(&counts[0], (unsigned long long)n_skip);
         if (n_repl) atomicAdd(&counts[1], (unsigned long long)n_repl);

@@ -173,6 +173,21 @@ def test_prefill_many_short_work_items(flashd_lib, shape):
     ok_status(flashd_lib)
 
 
+@pytest.mark.parametrize("d", [16, 256])
+@pytest.mark.parametrize("causal", [False, True])
+def test_perkey_hidden_sizes_of_the_paper(flashd_lib, d, causal):
+    """d = 16 and 256, the ends of the hidden sizes of Sec. V-A (fp32 and bf16 inputs)."""
+    sc = f32_scale(d)
+    q, k, v = synth.random_qkv(2, 3, 37, 91, d, seed=40 + d, dtype="f32")
+    want = oracle.attn_flashd(q, k, v, sc, causal)
+    got = flashd_lib.flashd_attn_fwd_f32(q.cuda(), k.cuda(), v.cuda(), sc, causal)
+    assert np.abs(got.double().cpu().numpy() - want).max() <= F32_MAX
+    q, k, v = synth.random_qkv(2, 3, 37, 91, d, seed=41 + d)
+    want = oracle.attn_naive(q, k, v, sc, causal)
+    got = flashd_lib.flashd_attn_fwd_perkey(q.cuda(), k.cuda(), v.cuda(), sc, causal)
+    check_bf16(got, want, d)
+
+
 def test_prefill_zero_scale_is_rejected(flashd_lib):
     q, k, v = synth.random_qkv(1, 1, 8, 8, 64, seed=1, device="cuda")
     with pytest.raises(flashd_lib.FlashdError) as ei:
