@@ -34,7 +34,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (c4: a batch-4 capture scaled by 16, traffic being
 # proportional to the bytes streamed).  Must be set back to None when that kernel changes.
-NCU_TRAFFIC_BYTES = {"c1": 38.1e6, "c2": 585.4e6, "c3": None, "c4": 34.49e9}
+NCU_TRAFFIC_BYTES = {"c1": 38.3e6, "c2": 591.1e6, "c3": None, "c4": 34.51e9}
 
 
 def f32(x: float) -> float:
@@ -400,10 +400,13 @@ def run_pwl_study(fd, synth, torch, device):
                       "workloads": out}), flush=True)
 
 
-def run_gqa(fd, synth, torch, device, peaks, steps):
+def run_gqa(fd, synth, torch, device, peaks, steps, batch=0):
     """Grouped-query decode: config 4 with its 32 query heads sharing 32/G K/V heads.  The K/V
     stream (the algorithmic bytes) shrinks by G, the arithmetic per K/V byte grows by G."""
     w4 = synth.WORKLOADS["c4"]
+    if batch > 0:
+        import dataclasses
+        w4 = dataclasses.replace(w4, B=batch)
     out = {}
     for G in (1, 4, 8):
         Hkv = w4.H // G
@@ -483,7 +486,7 @@ def main():
         run_pwl_study(fd, synth, torch, device)
         return
     if args.gqa:
-        run_gqa(fd, synth, torch, device, peaks, min(args.steps, 30))
+        run_gqa(fd, synth, torch, device, peaks, min(args.steps, 30), args.batch)
         return
 
     sampler = ClockSampler(local_rank)
