@@ -427,6 +427,26 @@ def run_gqa(fd, synth, torch, device, peaks, steps, batch=0):
                          "tflops": flops / (ms * 1e-3) / 1e12, "kv_gb": (k.numel() + v.numel()) * 2 / 1e9}
         del q, k, v, ws, o
         torch.cuda.empty_cache()
+    # config 4 itself with K and V stored as FP8-E4M3: half the bytes per key
+    g = torch.Generator(device=device).manual_seed(w4.seed + 99)
+    q = torch.randn(w4.B, w4.H, 1, w4.d, generator=g, device=device).to(torch.bfloat16)
+    k = torch.empty(w4.B, w4.H, w4.Nk, w4.d, dtype=torch.float8_e4m3fn, device=device)
+    v = torch.empty_like(k)
+    for b in range(w4.B):
+        k[b] = torch.randn(w4.H, w4.Nk, w4.d, generator=g, device=device).to(torch.float8_e4m3fn)
+        v[b] = torch.randn(w4.H, w4.Nk, w4.d, generator=g, device=device).to(torch.float8_e4m3fn)
+    sc = f32(w4.scale)
+    S = fd.flashd_splitk_num_splits(w4.B, w4.H, 1, w4.Nk, w4.d)
+    ws = torch.empty((w4.B, w4.H, 1, S, w4.d + 1), dtype=torch.float32, device=device)
+    o = torch.empty_like(q)
+    ms = time_gpu(lambda i: fd.flashd_attn_fwd_splitk_fp8kv(q, k, v, sc, S, workspace=ws, o=o), steps, 3, torch) / steps
+    alg = k.numel() + v.numel() + (q.numel() + o.numel()) * 2
+    out["fp8_kv"] = {"B": w4.B, "H": w4.H, "Nk": w4.Nk, "d": w4.d, "num_splits": S, "ms_per_step": ms,
+                     "gbs": alg / (ms * 1e-3) / 1e9, "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                     "frac_hbm_nominal": alg / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+                     "keys_per_s": w4.B * w4.H * w4.Nk / (ms * 1e-3), "kv_gb": (k.numel() + v.numel()) / 1e9}
+    del q, k, v, ws, o
+    torch.cuda.empty_cache()
     st, detail = fd.flashd_last_device_status()
     if st != 0:
         raise SystemExit(f"device status {st} {detail}")
@@ -448,7 +468,7 @@ def main():
     ap.add_argument("--pwl-study", action="store_true",
                     help="print the output error of the PWL / confined-range datapath model (Sec. IV-B) instead of timing")
     ap.add_argument("--gqa", action="store_true",
-                    help="time the grouped-query decode variant (config 4 with shared K/V heads) instead")
+                    help="time the decode variants (config 4 with shared K/V heads; config 4 with FP8-E4M3 K/V) instead")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the workload's batch size B (smaller case for profiler captures)")
     args = ap.parse_args()

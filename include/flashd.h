@@ -173,6 +173,25 @@ int flashd_attn_fwd_splitk(const void* q, const void* k, const void* v, void* o,
                            int num_splits, void* stream);
 
 /* ------------------------------------------------------------------------
+ * Split-K forward with K and V stored as FP8-E4M3 (the second number format of
+ * the paper's evaluation, Sec. V-A).  q and o stay bf16; k, v : [B,H,Nk,d] of
+ * one-byte E4M3 values (4 exponent bits, bias 7, 3 mantissa bits, no
+ * infinities: the "fn" variant), contiguous, 16-byte aligned.  Every element
+ * is widened exactly and the arithmetic is the fp32 arithmetic of
+ * flashd_splitk_partial: same function, same workspace layout, same combine,
+ * half the bytes per key.  A dequantisation scale of K folds into `scale`; one
+ * of V multiplies the output and is the caller's.  Other arguments, split
+ * rules and errors as flashd_splitk_partial / flashd_attn_fwd_splitk.       */
+int flashd_splitk_partial_fp8kv(const void* q, const void* k, const void* v,
+                                void* workspace, size_t workspace_bytes,
+                                int B, int H, int Nq, int Nk, int d, float scale,
+                                int num_splits, void* stream);
+int flashd_attn_fwd_splitk_fp8kv(const void* q, const void* k, const void* v, void* o,
+                                 void* workspace, size_t workspace_bytes,
+                                 int B, int H, int Nq, int Nk, int d, float scale,
+                                 int num_splits, void* stream);
+
+/* ------------------------------------------------------------------------
  * Grouped-query split-K forward (decode with shared K/V heads).
  * One query position, bf16 in, d = 128 or 64, non-causal.
  *

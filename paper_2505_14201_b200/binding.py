@@ -19,6 +19,7 @@ EXPORTED_SYMBOLS = (
     "flashd_splitk_workspace_bytes", "flashd_splitk_num_splits", "flashd_splitk_partial",
     "flashd_splitk_combine", "flashd_attn_fwd_splitk", "flashd_attn_fwd_splitk_static",
     "flashd_gqa_num_splits", "flashd_gqa_partial", "flashd_attn_fwd_gqa", "flashd_attn_fwd_pwl",
+    "flashd_splitk_partial_fp8kv", "flashd_attn_fwd_splitk_fp8kv",
     "flashd_attn_fwd_host", "flashd_skip_stats", "flashd_last_device_status", "flashd_status_string", "flashd_version", "flashd_launch_count",
 )
 
@@ -66,6 +67,8 @@ def lib() -> ctypes.CDLL:
             L.flashd_gqa_num_splits.argtypes = [ci, ci, ci, ci, ci]
             L.flashd_gqa_partial.argtypes = [vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_attn_fwd_gqa.argtypes = [vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
+            L.flashd_splitk_partial_fp8kv.argtypes = [vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
+            L.flashd_attn_fwd_splitk_fp8kv.argtypes = [vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_attn_fwd_splitk_static.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_skip_stats.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, cf, cf, cf, cf, vp]
             L.flashd_attn_fwd_host.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp]
@@ -307,6 +310,37 @@ def flashd_attn_fwd_gqa(q, k, v, scale, num_splits=0, workspace=None, o=None, st
     _check(lib().flashd_attn_fwd_gqa(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(workspace),
                                      workspace.numel() * workspace.element_size(), B, Hkv, G, Nk, d,
                                      float(scale), int(num_splits), _stream_ptr(stream)), "flashd_attn_fwd_gqa")
+    return o
+
+
+def flashd_splitk_partial_fp8kv(q, k, v, scale, num_splits, workspace=None, stream=None):
+    """Partial states of the split-K forward with E4M3 K/V (``torch.float8_e4m3fn``), q bf16."""
+    import torch
+    B, H, Nq, Nk, d = _dims(q, k, v)
+    if workspace is None:
+        workspace = torch.empty((B, H, Nq, num_splits, d + 1), dtype=torch.float32, device=q.device)
+    _check(lib().flashd_splitk_partial_fp8kv(_ptr(q), _ptr(k), _ptr(v), _ptr(workspace),
+                                             workspace.numel() * workspace.element_size(), B, H, Nq, Nk, d,
+                                             float(scale), int(num_splits), _stream_ptr(stream)),
+           "flashd_splitk_partial_fp8kv")
+    return workspace
+
+
+def flashd_attn_fwd_splitk_fp8kv(q, k, v, scale, num_splits=0, workspace=None, o=None, stream=None):
+    """Split-K forward with E4M3 K/V: q, o bf16 ``[B,H,Nq,d]``; k, v ``torch.float8_e4m3fn``."""
+    import torch
+    B, H, Nq, Nk, d = _dims(q, k, v)
+    if q.dtype != torch.bfloat16 or k.dtype != torch.float8_e4m3fn or v.dtype != torch.float8_e4m3fn:
+        raise ValueError("expected bf16 q and float8_e4m3fn k, v")
+    S = num_splits if num_splits > 0 else flashd_splitk_num_splits(B, H, Nq, Nk, d)
+    if workspace is None:
+        workspace = torch.empty((B, H, Nq, max(S, 1), d + 1), dtype=torch.float32, device=q.device)
+    if o is None:
+        o = torch.empty_like(q)
+    _check(lib().flashd_attn_fwd_splitk_fp8kv(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(workspace),
+                                              workspace.numel() * workspace.element_size(), B, H, Nq, Nk, d,
+                                              float(scale), int(num_splits), _stream_ptr(stream)),
+           "flashd_attn_fwd_splitk_fp8kv")
     return o
 
 

@@ -179,15 +179,15 @@ bool fill_table(int n, const float* x, const float* y, int* n_out, float* xs, fl
     return true;
 }
 
-template <int D>
+template <int D, int KVB = 2>
 int launch_partial(const void* q, const void* k, const void* v, void* ws, long long rows, int Nq, int Nk,
                    float scale, int num_splits, cudaStream_t stream) {
-    using C = DecodeCfg<D>;
+    using C = DecodeCfg<D, KVB>;
     static bool attr_set[64] = {false};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FLASHD_ERR_CUDA;
     if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(splitk_partial_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(splitk_partial_kernel<D, KVB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  C::kSmemBytes) != cudaSuccess)
             return FLASHD_ERR_CUDA;
         attr_set[dev] = true;
@@ -196,9 +196,9 @@ int launch_partial(const void* q, const void* k, const void* v, void* ws, long l
     if (sms <= 0) return FLASHD_ERR_CUDA;
     const long long items = rows * num_splits;
     const int grid = (int)(items < sms ? items : sms);
-    splitk_partial_kernel<D><<<grid, C::kThreads, C::kSmemBytes, stream>>>(
-        static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
-        static_cast<const __nv_bfloat16*>(v), static_cast<float*>(ws), rows, Nq, Nk, scale * kLog2e, num_splits);
+    splitk_partial_kernel<D, KVB><<<grid, C::kThreads, C::kSmemBytes, stream>>>(
+        static_cast<const __nv_bfloat16*>(q), static_cast<const unsigned char*>(k),
+        static_cast<const unsigned char*>(v), static_cast<float*>(ws), rows, Nq, Nk, scale * kLog2e, num_splits);
     return after_launch();
 }
 
@@ -402,6 +402,30 @@ int flashd_attn_fwd_splitk(const void* q, const void* k, const void* v, void* o,
     if (num_splits <= 0) num_splits = flashd_splitk_num_splits(B, H, Nq, Nk, d);
     if (!workspace) return FLASHD_ERR_NULL;
     int st = flashd_splitk_partial(q, k, v, workspace, workspace_bytes, B, H, Nq, Nk, d, scale, num_splits, stream);
+    if (st != FLASHD_OK) return st;
+    return flashd_splitk_combine(workspace, o, nullptr, B, H, Nq, d, num_splits, FLASHD_BF16, stream);
+}
+
+int flashd_splitk_partial_fp8kv(const void* q, const void* k, const void* v, void* workspace, size_t workspace_bytes,
+                                int B, int H, int Nq, int Nk, int d, float scale, int num_splits, void* stream) {
+    const int st = check_common(q, k, v, workspace, B, H, Nq, Nk, d, scale);
+    if (st != FLASHD_OK) return st;
+    if (d != 128 && d != 64) return FLASHD_ERR_UNSUPPORTED;
+    const int cs = check_splits(Nk, num_splits);
+    if (cs != FLASHD_OK) return cs;
+    if (workspace_bytes < flashd_splitk_workspace_bytes(B, H, Nq, d, num_splits)) return FLASHD_ERR_WORKSPACE;
+    const long long rows = (long long)B * H * Nq;
+    if (d == 128) return launch_partial<128, 1>(q, k, v, workspace, rows, Nq, Nk, scale, num_splits, as_stream(stream));
+    return launch_partial<64, 1>(q, k, v, workspace, rows, Nq, Nk, scale, num_splits, as_stream(stream));
+}
+
+int flashd_attn_fwd_splitk_fp8kv(const void* q, const void* k, const void* v, void* o, void* workspace,
+                                 size_t workspace_bytes, int B, int H, int Nq, int Nk, int d, float scale,
+                                 int num_splits, void* stream) {
+    if (!o || !workspace) return FLASHD_ERR_NULL;
+    if (num_splits <= 0) num_splits = flashd_splitk_num_splits(B, H, Nq, Nk, d);
+    const int st = flashd_splitk_partial_fp8kv(q, k, v, workspace, workspace_bytes, B, H, Nq, Nk, d, scale,
+                                               num_splits, stream);
     if (st != FLASHD_OK) return st;
     return flashd_splitk_combine(workspace, o, nullptr, B, H, Nq, d, num_splits, FLASHD_BF16, stream);
 }

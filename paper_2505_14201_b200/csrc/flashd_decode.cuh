@@ -13,23 +13,31 @@
 // same super-key step in the one-multiplier form of Sec. IV-A:
 //     o <- o + (o_p - o) W,  L <- L_p - ln W.
 // L is kept in log2 units inside the kernels and written in natural log.
+//
+// K and V are stored either as bf16 (KVB = 2 bytes per element) or as FP8-E4M3
+// (KVB = 1; the second number format of Sec. V-A).  E4M3 rows are half as long, so
+// the same bytes per ring stage hold twice the keys; every element is widened
+// exactly (e4m3 -> f16 -> f32) and all arithmetic stays in fp32, as for bf16.
 #pragma once
+
+#include <cuda_fp16.h>
 
 #include "flashd_common.cuh"
 
 namespace flashd {
 
-template <int D>
+template <int D, int KVB = 2>
 struct DecodeCfg {
-    static constexpr int kChunk = 8192 / D;                  // keys per ring stage (16 KB of K, 16 KB of V)
+    static constexpr int kChunk = 16384 / (D * KVB);         // keys per ring stage (16 KB of K, 16 KB of V)
     static constexpr int kStages = 5;
     static constexpr int kConsumerWarps = 8;
     static constexpr int kThreads = (kConsumerWarps + 1) * 32;
-    static constexpr int kLanesPerRow = D / 8;               // 16-byte slices per key row
+    static constexpr int kElems = 16 / KVB;                  // elements of a 16-byte slice
+    static constexpr int kLanesPerRow = D / kElems;          // 16-byte slices per key row
     static constexpr int kRowsPerWarp = 32 / kLanesPerRow;
     static constexpr int kGroups = kConsumerWarps * kRowsPerWarp;
     static constexpr int kKeysPerGroup = kChunk / kGroups;   // = 4
-    static constexpr int kTileBytes = kChunk * D * 2;
+    static constexpr int kTileBytes = kChunk * D * KVB;
     static constexpr int kStageBytes = 2 * kTileBytes;
     static constexpr int kMergeFloats = kGroups * (D + 1);
     static constexpr int kSmemBytes = kStages * kStageBytes + kMergeFloats * 4 + 256;
@@ -57,12 +65,34 @@ __device__ __forceinline__ float superkey_weight(float& L_acc, float Lp) {
     return W;
 }
 
-template <int D>
-__global__ void __launch_bounds__(DecodeCfg<D>::kThreads, 1)
-splitk_partial_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
-                      const __nv_bfloat16* __restrict__ v, float* __restrict__ workspace,
+// One 16-byte slice of a K or V row widened to fp32: 8 bf16 or 16 e4m3 elements.
+template <int KVB> __device__ __forceinline__ void widen_slice(const uint4& raw, float (&f)[16 / KVB]);
+template <> __device__ __forceinline__ void widen_slice<2>(const uint4& raw, float (&f)[8]) {
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { f[2 * e] = bf16_lo(w[e]); f[2 * e + 1] = bf16_hi(w[e]); }
+}
+template <> __device__ __forceinline__ void widen_slice<1>(const uint4& raw, float (&f)[16]) {
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        uint32_t h01, h23;      // two f16x2 pairs: bytes 0,1 and bytes 2,3 of the word
+        asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\t"
+            "cvt.rn.f16x2.e4m3x2 %0, lo;\n\tcvt.rn.f16x2.e4m3x2 %1, hi;\n\t}"
+            : "=r"(h01), "=r"(h23) : "r"(w[e]));
+        const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&h01));
+        const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&h23));
+        f[4 * e] = a.x; f[4 * e + 1] = a.y; f[4 * e + 2] = b.x; f[4 * e + 3] = b.y;
+    }
+}
+
+template <int D, int KVB>
+__global__ void __launch_bounds__(DecodeCfg<D, KVB>::kThreads, 1)
+splitk_partial_kernel(const __nv_bfloat16* __restrict__ q, const unsigned char* __restrict__ k,
+                      const unsigned char* __restrict__ v, float* __restrict__ workspace,
                       long long rows, int Nq, int Nk, float scale_log2e, int num_splits) {
-    using C = DecodeCfg<D>;
+    using C = DecodeCfg<D, KVB>;
+    constexpr int EL = C::kElems;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     unsigned char* ring = smem_raw;
     float* merge = reinterpret_cast<float*>(smem_raw + C::kStages * C::kStageBytes);
@@ -95,18 +125,18 @@ splitk_partial_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
             const long long bh = row / Nq;
             const int k0 = split * per_split;
             const int k1 = min(k0 + per_split, Nk);
-            const __nv_bfloat16* kb = k + (bh * Nk) * (long long)D;
-            const __nv_bfloat16* vb = v + (bh * Nk) * (long long)D;
+            const unsigned char* kb = k + (bh * Nk) * (long long)(D * KVB);
+            const unsigned char* vb = v + (bh * Nk) * (long long)(D * KVB);
             for (int c0 = k0; c0 < k1; c0 += C::kChunk, ++it) {
                 const int stage = it % C::kStages;
                 const uint32_t round = it / C::kStages;
                 if (round > 0 && !mbar_wait(&empty[stage], (round - 1) & 1, kWaitDecEmpty)) return;
                 const int nk = min(C::kChunk, k1 - c0);
-                const uint32_t bytes = (uint32_t)nk * D * 2;
+                const uint32_t bytes = (uint32_t)nk * D * KVB;
                 unsigned char* dst = ring + stage * C::kStageBytes;
                 mbar_arrive_expect_tx(&full[stage], 2 * bytes);
-                bulk_load(dst, kb + (long long)c0 * D, bytes, &full[stage]);
-                bulk_load(dst + C::kTileBytes, vb + (long long)c0 * D, bytes, &full[stage]);
+                bulk_load(dst, kb + (long long)c0 * (D * KVB), bytes, &full[stage]);
+                bulk_load(dst + C::kTileBytes, vb + (long long)c0 * (D * KVB), bytes, &full[stage]);
             }
         }
         return;
@@ -123,19 +153,20 @@ splitk_partial_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
         const int k0 = split * per_split;
         const int k1 = min(k0 + per_split, Nk);
 
-        float qf[8];
-        {
-            const uint4 qw = *reinterpret_cast<const uint4*>(q + row * D + sl * 8);
+        float qf[EL];
+#pragma unroll
+        for (int h = 0; h < EL / 8; ++h) {
+            const uint4 qw = *reinterpret_cast<const uint4*>(q + row * D + sl * EL + h * 8);
             const uint32_t w[4] = {qw.x, qw.y, qw.z, qw.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                qf[2 * e] = bf16_lo(w[e]) * scale_log2e;
-                qf[2 * e + 1] = bf16_hi(w[e]) * scale_log2e;
+                qf[8 * h + 2 * e] = bf16_lo(w[e]) * scale_log2e;
+                qf[8 * h + 2 * e + 1] = bf16_hi(w[e]) * scale_log2e;
             }
         }
-        float of[8];
+        float of[EL];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) of[e] = 0.f;
+        for (int e = 0; e < EL; ++e) of[e] = 0.f;
         float L = -INFINITY;
 
         for (int c0 = k0; c0 < k1; c0 += C::kChunk, ++it) {
@@ -152,14 +183,12 @@ splitk_partial_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
             for (int m = 0; m < C::kKeysPerGroup; ++m) {
                 const int r = g + C::kGroups * m;
                 valid[m] = r < nk;
-                const uint4 kw = *reinterpret_cast<const uint4*>(ks + (r * D + sl * 8) * 2);
-                const uint32_t w[4] = {kw.x, kw.y, kw.z, kw.w};
+                const uint4 kw = *reinterpret_cast<const uint4*>(ks + r * (D * KVB) + sl * 16);
+                float kf[EL];
+                widen_slice<KVB>(kw, kf);
                 float acc = 0.f;
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    acc = fmaf(qf[2 * e], bf16_lo(w[e]), acc);
-                    acc = fmaf(qf[2 * e + 1], bf16_hi(w[e]), acc);
-                }
+                for (int e = 0; e < EL; ++e) acc = fmaf(qf[e], kf[e], acc);
                 s[m] = acc;
             }
 #pragma unroll
@@ -184,19 +213,17 @@ splitk_partial_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
                 const float alpha = e_old * inv;          // = 1 - W = exp(L_old - L_new)
                 L = ref + lg2(l);                          // L_new
 #pragma unroll
-                for (int e = 0; e < 8; ++e) of[e] *= alpha;
+                for (int e = 0; e < EL; ++e) of[e] *= alpha;
 #pragma unroll
                 for (int m = 0; m < C::kKeysPerGroup; ++m) {
                     const int r = g + C::kGroups * m;
                     const float P = p[m] * inv;            // = exp(s_j - L_new)
-                    uint4 vw = *reinterpret_cast<const uint4*>(vs + (r * D + sl * 8) * 2);
+                    uint4 vw = *reinterpret_cast<const uint4*>(vs + r * (D * KVB) + sl * 16);
                     if (!valid[m]) vw = make_uint4(0u, 0u, 0u, 0u);
-                    const uint32_t w[4] = {vw.x, vw.y, vw.z, vw.w};
+                    float vf[EL];
+                    widen_slice<KVB>(vw, vf);
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        of[2 * e] = fmaf(P, bf16_lo(w[e]), of[2 * e]);
-                        of[2 * e + 1] = fmaf(P, bf16_hi(w[e]), of[2 * e + 1]);
-                    }
+                    for (int e = 0; e < EL; ++e) of[e] = fmaf(P, vf[e], of[e]);
                 }
             }
             __syncwarp();
@@ -208,7 +235,7 @@ splitk_partial_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
         {
             float* mine = merge + g * (D + 1);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) mine[sl * 8 + e] = of[e];
+            for (int e = 0; e < EL; ++e) mine[sl * EL + e] = of[e];
             if (sl == 0) mine[D] = L;
         }
         __syncwarp();
