@@ -192,21 +192,26 @@ int flashd_attn_fwd_splitk_fp8kv(const void* q, const void* k, const void* v, vo
                                  int num_splits, void* stream);
 
 /* ------------------------------------------------------------------------
- * Grouped-query split-K forward (decode with shared K/V heads).
- * One query position, bf16 in, d = 128 or 64, non-causal.
+ * Grouped-query split-K forward (decode with shared K/V heads, one or a few
+ * query positions).  bf16 in, d = 128 or 64.
  *
  * G consecutive query heads attend to the same K/V head: query head
  * h = hkv*G + g reads k[b,hkv], v[b,hkv].  The attention function of every
  * query head is unchanged (Eq. (out-final)/(w-last) per head); only the data
  * movement differs: each split's K and V rows are read from device memory
  * once and serve all G queries.
- *   q, o : [B, Hkv*G, 1, d] contiguous;  k, v : [B, Hkv, Nk, d] contiguous.
- *   1 <= G <= FLASHD_MAX_GROUP (larger: FLASHD_ERR_UNSUPPORTED).
- * flashd_gqa_partial writes the partial states [B, Hkv*G, 1, num_splits, d+1]
- * fp32 exactly as flashd_splitk_partial does for a [B, Hkv*G, 1, d] query
- * tensor, so flashd_splitk_combine(workspace, o, lse, B, Hkv*G, 1, d, ...)
- * finishes it; flashd_attn_fwd_gqa queues both (bf16 output).  Workspace
- * size: flashd_splitk_workspace_bytes(B, Hkv*G, 1, d, num_splits); ownership,
+ *   q, o : [B, Hkv*G, Nq, d] contiguous;  k, v : [B, Hkv, Nk, d] contiguous.
+ *   G >= 1, Nq >= 1, G*Nq <= FLASHD_MAX_GROUP (larger: FLASHD_ERR_UNSUPPORTED).
+ * The Nq query positions are the LAST Nq positions of the Nk-key sequence
+ * (a decode step over several tokens: speculative or chunked decoding).
+ * causal != 0: query position iq sees keys 0 .. Nk-Nq+iq (needs Nq <= Nk);
+ * causal == 0: every query sees all Nk keys.
+ * flashd_gqa_partial writes the partial states [B, Hkv*G, Nq, num_splits, d+1]
+ * fp32 exactly as flashd_splitk_partial does for a [B, Hkv*G, Nq, d] query
+ * tensor (a split with no visible key for a row is written as empty), so
+ * flashd_splitk_combine(workspace, o, lse, B, Hkv*G, Nq, d, ...) finishes
+ * it; flashd_attn_fwd_gqa queues both (bf16 output).  Workspace size:
+ * flashd_splitk_workspace_bytes(B, Hkv*G, Nq, d, num_splits); ownership,
  * alignment, split rules and errors as for the split-K calls above.
  * flashd_gqa_num_splits returns the library's split count (num_splits <= 0
  * in flashd_attn_fwd_gqa selects it).                                      */
@@ -214,11 +219,11 @@ int flashd_attn_fwd_splitk_fp8kv(const void* q, const void* k, const void* v, vo
 int flashd_gqa_num_splits(int B, int Hkv, int G, int Nk, int d);
 int flashd_gqa_partial(const void* q, const void* k, const void* v,
                        void* workspace, size_t workspace_bytes,
-                       int B, int Hkv, int G, int Nk, int d, float scale,
+                       int B, int Hkv, int G, int Nq, int Nk, int d, float scale, int causal,
                        int num_splits, void* stream);
 int flashd_attn_fwd_gqa(const void* q, const void* k, const void* v, void* o,
                         void* workspace, size_t workspace_bytes,
-                        int B, int Hkv, int G, int Nk, int d, float scale,
+                        int B, int Hkv, int G, int Nq, int Nk, int d, float scale, int causal,
                         int num_splits, void* stream);
 
 /* ------------------------------------------------------------------------

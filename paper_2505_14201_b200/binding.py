@@ -65,8 +65,8 @@ def lib() -> ctypes.CDLL:
             L.flashd_attn_fwd_pwl.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, ci,
                                               ci, fp, fp, ci, fp, fp, cf, cf, ci, vp]
             L.flashd_gqa_num_splits.argtypes = [ci, ci, ci, ci, ci]
-            L.flashd_gqa_partial.argtypes = [vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
-            L.flashd_attn_fwd_gqa.argtypes = [vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
+            L.flashd_gqa_partial.argtypes = [vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, ci, cf, ci, ci, vp]
+            L.flashd_attn_fwd_gqa.argtypes = [vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, ci, cf, ci, ci, vp]
             L.flashd_splitk_partial_fp8kv.argtypes = [vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_attn_fwd_splitk_fp8kv.argtypes = [vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_attn_fwd_splitk_static.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, ci, vp]
@@ -277,39 +277,42 @@ def _gqa_dims(q, k, v):
             raise ValueError("q, k, v must be contiguous [B, H, N, d] tensors")
     B, Hq, Nq, d = q.shape
     Bk, Hkv, Nk, dk = k.shape
-    if Nq != 1 or Bk != B or dk != d or tuple(v.shape) != tuple(k.shape) or Hkv == 0 or Hq % Hkv != 0:
+    if Bk != B or dk != d or tuple(v.shape) != tuple(k.shape) or Hkv == 0 or Hq % Hkv != 0:
         raise ValueError(f"grouped-query shapes do not match: q {tuple(q.shape)} k {tuple(k.shape)} v {tuple(v.shape)}")
-    return B, Hkv, Hq // Hkv, Nk, d
+    return B, Hkv, Hq // Hkv, Nq, Nk, d
 
 
 def flashd_gqa_num_splits(B, Hkv, G, Nk, d) -> int:
     return int(lib().flashd_gqa_num_splits(B, Hkv, G, Nk, d))
 
 
-def flashd_gqa_partial(q, k, v, scale, num_splits, workspace=None, stream=None):
-    """Partial states ``[B,Hkv*G,1,num_splits,d+1]`` fp32 of the grouped-query split-K forward."""
+def flashd_gqa_partial(q, k, v, scale, num_splits, causal=False, workspace=None, stream=None):
+    """Partial states ``[B,Hkv*G,Nq,num_splits,d+1]`` fp32 of the grouped-query split-K forward."""
     import torch
-    B, Hkv, G, Nk, d = _gqa_dims(q, k, v)
+    B, Hkv, G, Nq, Nk, d = _gqa_dims(q, k, v)
     if workspace is None:
-        workspace = torch.empty((B, Hkv * G, 1, num_splits, d + 1), dtype=torch.float32, device=q.device)
+        workspace = torch.empty((B, Hkv * G, Nq, num_splits, d + 1), dtype=torch.float32, device=q.device)
     _check(lib().flashd_gqa_partial(_ptr(q), _ptr(k), _ptr(v), _ptr(workspace),
-                                    workspace.numel() * workspace.element_size(), B, Hkv, G, Nk, d,
-                                    float(scale), int(num_splits), _stream_ptr(stream)), "flashd_gqa_partial")
+                                    workspace.numel() * workspace.element_size(), B, Hkv, G, Nq, Nk, d,
+                                    float(scale), int(bool(causal)), int(num_splits), _stream_ptr(stream)),
+           "flashd_gqa_partial")
     return workspace
 
 
-def flashd_attn_fwd_gqa(q, k, v, scale, num_splits=0, workspace=None, o=None, stream=None):
-    """Grouped-query split-K forward: q ``[B,Hkv*G,1,d]``, k/v ``[B,Hkv,Nk,d]``."""
+def flashd_attn_fwd_gqa(q, k, v, scale, num_splits=0, causal=False, workspace=None, o=None, stream=None):
+    """Grouped-query split-K forward: q ``[B,Hkv*G,Nq,d]`` (the last Nq positions of the
+    sequence; ``causal`` masks among them), k/v ``[B,Hkv,Nk,d]``; G*Nq <= 8."""
     import torch
-    B, Hkv, G, Nk, d = _gqa_dims(q, k, v)
+    B, Hkv, G, Nq, Nk, d = _gqa_dims(q, k, v)
     S = num_splits if num_splits > 0 else flashd_gqa_num_splits(B, Hkv, G, Nk, d)
     if workspace is None:
-        workspace = torch.empty((B, Hkv * G, 1, max(S, 1), d + 1), dtype=torch.float32, device=q.device)
+        workspace = torch.empty((B, Hkv * G, Nq, max(S, 1), d + 1), dtype=torch.float32, device=q.device)
     if o is None:
         o = torch.empty_like(q)
     _check(lib().flashd_attn_fwd_gqa(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(workspace),
-                                     workspace.numel() * workspace.element_size(), B, Hkv, G, Nk, d,
-                                     float(scale), int(num_splits), _stream_ptr(stream)), "flashd_attn_fwd_gqa")
+                                     workspace.numel() * workspace.element_size(), B, Hkv, G, Nq, Nk, d,
+                                     float(scale), int(bool(causal)), int(num_splits), _stream_ptr(stream)),
+           "flashd_attn_fwd_gqa")
     return o
 
 

@@ -203,8 +203,8 @@ int launch_partial(const void* q, const void* k, const void* v, void* ws, long l
 }
 
 template <int D>
-int launch_gqa_partial(const void* q, const void* k, const void* v, void* ws, int BHkv, int G, int Nk, float scale,
-                       int num_splits, cudaStream_t stream) {
+int launch_gqa_partial(const void* q, const void* k, const void* v, void* ws, int BHkv, int R, int Nq, int causal,
+                       int Nk, float scale, int num_splits, cudaStream_t stream) {
     using C = GqaCfg<D>;
     CUtensorMap mk, mv;
     if (!make_map(&mk, k, BHkv, Nk, D) || !make_map(&mv, v, BHkv, Nk, D)) return FLASHD_ERR_CUDA;
@@ -222,8 +222,8 @@ int launch_gqa_partial(const void* q, const void* k, const void* v, void* ws, in
     const long long items = (long long)BHkv * num_splits;
     const int grid = (int)(items < sms ? items : sms);
     gqa_partial_kernel<D><<<grid, C::kThreads, C::kSmemBytes, stream>>>(
-        mk, mv, static_cast<const __nv_bfloat16*>(q), static_cast<float*>(ws), BHkv, G, Nk, scale * kLog2e,
-        num_splits);
+        mk, mv, static_cast<const __nv_bfloat16*>(q), static_cast<float*>(ws), BHkv, R, Nq, causal, Nk,
+        scale * kLog2e, num_splits);
     return after_launch();
 }
 
@@ -436,27 +436,35 @@ int flashd_gqa_num_splits(int B, int Hkv, int G, int Nk, int d) {
 }
 
 int flashd_gqa_partial(const void* q, const void* k, const void* v, void* workspace, size_t workspace_bytes, int B,
-                       int Hkv, int G, int Nk, int d, float scale, int num_splits, void* stream) {
-    if (G < 1 || G > FLASHD_MAX_GROUP) return G < 1 ? FLASHD_ERR_SHAPE : FLASHD_ERR_UNSUPPORTED;
-    const int st = check_common(q, k, v, workspace, B, Hkv, 1, Nk, d, scale);
+                       int Hkv, int G, int Nq, int Nk, int d, float scale, int causal, int num_splits,
+                       void* stream) {
+    if (G < 1 || Nq < 1) return FLASHD_ERR_SHAPE;
+    if ((long long)G * Nq > FLASHD_MAX_GROUP) return FLASHD_ERR_UNSUPPORTED;
+    if (causal && Nq > Nk) return FLASHD_ERR_SHAPE;
+    const int st = check_common(q, k, v, workspace, B, Hkv, Nq, Nk, d, scale);
     if (st != FLASHD_OK) return st;
     if (d != 128 && d != 64) return FLASHD_ERR_UNSUPPORTED;
     const int cs = check_splits(Nk, num_splits);
     if (cs != FLASHD_OK) return cs;
     if ((long long)B * Hkv * G > 0x7fffffffLL / FLASHD_MAX_SPLITS) return FLASHD_ERR_SHAPE;
-    if (workspace_bytes < flashd_splitk_workspace_bytes(B, Hkv * G, 1, d, num_splits)) return FLASHD_ERR_WORKSPACE;
+    if (workspace_bytes < flashd_splitk_workspace_bytes(B, Hkv * G, Nq, d, num_splits)) return FLASHD_ERR_WORKSPACE;
     const int BHkv = B * Hkv;
-    if (d == 128) return launch_gqa_partial<128>(q, k, v, workspace, BHkv, G, Nk, scale, num_splits, as_stream(stream));
-    return launch_gqa_partial<64>(q, k, v, workspace, BHkv, G, Nk, scale, num_splits, as_stream(stream));
+    const int R = G * Nq;
+    const int cz = causal ? 1 : 0;
+    if (d == 128)
+        return launch_gqa_partial<128>(q, k, v, workspace, BHkv, R, Nq, cz, Nk, scale, num_splits, as_stream(stream));
+    return launch_gqa_partial<64>(q, k, v, workspace, BHkv, R, Nq, cz, Nk, scale, num_splits, as_stream(stream));
 }
 
 int flashd_attn_fwd_gqa(const void* q, const void* k, const void* v, void* o, void* workspace, size_t workspace_bytes,
-                        int B, int Hkv, int G, int Nk, int d, float scale, int num_splits, void* stream) {
+                        int B, int Hkv, int G, int Nq, int Nk, int d, float scale, int causal, int num_splits,
+                        void* stream) {
     if (!o || !workspace) return FLASHD_ERR_NULL;
     if (num_splits <= 0) num_splits = flashd_gqa_num_splits(B, Hkv, G, Nk, d);
-    const int st = flashd_gqa_partial(q, k, v, workspace, workspace_bytes, B, Hkv, G, Nk, d, scale, num_splits, stream);
+    const int st = flashd_gqa_partial(q, k, v, workspace, workspace_bytes, B, Hkv, G, Nq, Nk, d, scale, causal,
+                                      num_splits, stream);
     if (st != FLASHD_OK) return st;
-    return flashd_splitk_combine(workspace, o, nullptr, B, Hkv * G, 1, d, num_splits, FLASHD_BF16, stream);
+    return flashd_splitk_combine(workspace, o, nullptr, B, Hkv * G, Nq, d, num_splits, FLASHD_BF16, stream);
 }
 
 int flashd_attn_fwd_splitk_static(const void* q, const void* k, const void* v, void* o, int B, int H, int Nq,

@@ -1,4 +1,6 @@
-// Grouped-query split-K FLASH-D decode: G query heads share one K/V head.
+// Grouped-query split-K FLASH-D decode: G query heads share one K/V head, and
+// each may carry a few query positions (the last Nq positions of the sequence,
+// causal among themselves): R = G*Nq <= 8 query rows per K/V head.
 //
 // One work item = (batch, K/V head, split).  The split's K and V rows cross HBM
 // once and serve all G queries of the group, so the kernel is bound by the same
@@ -73,8 +75,8 @@ __device__ __forceinline__ void mma_rows8(float& d0, float& d1, uint32_t a0, uin
 template <int D>
 __global__ void __launch_bounds__(GqaCfg<D>::kThreads, 1)
 gqa_partial_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                   const __nv_bfloat16* __restrict__ q, float* __restrict__ workspace, int BHkv, int G, int Nk,
-                   float scale_log2e, int num_splits) {
+                   const __nv_bfloat16* __restrict__ q, float* __restrict__ workspace, int BHkv, int R, int Nq,
+                   int causal, int Nk, float scale_log2e, int num_splits) {
     using C = GqaCfg<D>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // swizzle atoms: 1 KB
@@ -124,7 +126,10 @@ gqa_partial_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     }
 
     // ---------------------------------------------------------- consumers
-    const int grow = lane >> 2;            // query of the group this lane's accumulator rows belong to
+    const int grow = lane >> 2;            // query row (head g, position iq: grow = g*Nq + iq) of this lane's accumulators
+    // keys [0, row_lim) are visible to the row: all of them, or, causal, up to the row's own
+    // position Nk - Nq + iq (the queries are the last Nq positions of the sequence)
+    const int row_lim = causal ? Nk - Nq + (grow % Nq) + 1 : Nk;
     const int quad = lane & 3;
     constexpr int KS = D / 16;             // k-steps of the score product = pairs of output column tiles
     // shared-memory offsets of this lane's matrix rows (within a K or V tile)
@@ -145,12 +150,12 @@ gqa_partial_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         // Q fragments of the group: row grow, columns 16 ks + 2 quad (+8)
         uint32_t qa0[KS], qa2[KS];
         {
-            const __nv_bfloat16* qrow = q + ((long long)bh * G + grow) * D;
+            const __nv_bfloat16* qrow = q + ((long long)bh * R + grow) * D;
 #pragma unroll
             for (int ks = 0; ks < KS; ++ks) {
                 qa0[ks] = 0u;
                 qa2[ks] = 0u;
-                if (grow < G) {
+                if (grow < R) {
                     qa0[ks] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * quad);
                     qa2[ks] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + 2 * quad);
                 }
@@ -186,12 +191,15 @@ gqa_partial_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
 #pragma unroll
                     for (int e = 0; e < 2; ++e) {
                         const int key = c0 + warp * 16 + nt * 8 + 2 * quad + e;
-                        s[nt][e] = key < k1 ? s[nt][e] * scale_log2e : -INFINITY;
+                        s[nt][e] = key < min(k1, row_lim) ? s[nt][e] * scale_log2e : -INFINITY;
                         mx = fmaxf(mx, s[nt][e]);
                     }
                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                const float ref = fmaxf(L, mx);          // finite: the warp's first key is inside the split
+                // -inf only while the row has seen no visible key yet (causal rows at the end of
+                // the sequence): the step then leaves the empty state as it is
+                const float ref_raw = fmaxf(L, mx);
+                const float ref = ref_raw == -INFINITY ? 0.f : ref_raw;
                 const float e_old = ex2(L - ref);
                 float p[2][2];
                 float sum = 0.f;
@@ -202,9 +210,9 @@ gqa_partial_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
                 sum += __shfl_xor_sync(0xffffffffu, sum, 1);
                 sum += __shfl_xor_sync(0xffffffffu, sum, 2);
                 const float l = e_old + sum;
-                const float inv = rcp(l);
+                const float inv = l > 0.f ? rcp(l) : 0.f;
                 const float alpha = e_old * inv;         // = exp(L_old - L_new)
-                L = ref + lg2(l);
+                L = l > 0.f ? ref + lg2(l) : -INFINITY;
                 const uint32_t pa0 = pack_bf16x2(p[0][0] * inv, p[0][1] * inv);   // keys 2 quad, +1
                 const uint32_t pa2 = pack_bf16x2(p[1][0] * inv, p[1][1] * inv);   // keys 8 + 2 quad, +1
 #pragma unroll
@@ -237,7 +245,7 @@ gqa_partial_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         __syncwarp();
         if (lane == 0) mbar_arrive(merge_ready);
         if (!mbar_wait(merge_ready, item_idx & 1, kWaitGqaMergeReady)) return;
-        for (int idx = threadIdx.x; idx < G * D; idx += C::kConsumerWarps * 32) {
+        for (int idx = threadIdx.x; idx < R * D; idx += C::kConsumerWarps * 32) {
             const int gq = idx / D;
             const int c = idx - gq * D;
             float L_acc = -INFINITY, o_acc = 0.f;
@@ -247,7 +255,7 @@ gqa_partial_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
                 const float W = superkey_weight(L_acc, st[D]);
                 o_acc = fmaf(st[c] - o_acc, W, o_acc);
             }
-            float* wp = workspace + (((long long)bh * G + gq) * num_splits + split) * (long long)(D + 1);
+            float* wp = workspace + (((long long)bh * R + gq) * num_splits + split) * (long long)(D + 1);
             wp[c] = o_acc;
             if (c == 0) wp[D] = L_acc * kLn2;
         }

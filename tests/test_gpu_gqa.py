@@ -75,6 +75,50 @@ def test_gqa_shapes(flashd_lib, shape):
         assert np.abs(pre.double().cpu().numpy() - wantp).max() <= 1e-2
 
 
+MULTI_Q_SHAPES = [
+    # B, Hkv, G, Nq, Nk, d, S, causal
+    (1, 2, 2, 4, 500, 128, 3, True),
+    (2, 2, 4, 2, 1000, 128, 4, True),
+    (1, 1, 1, 8, 100, 64, 2, True),
+    (1, 2, 2, 3, 300, 128, 2, False),      # G*Nq = 6, no mask among the positions
+    (1, 1, 2, 4, 4, 64, 1, True),          # Nk = Nq: the first position sees one key
+    (1, 1, 1, 8, 9, 64, 8, True),          # 2 keys per split: most splits are empty for the early positions
+    (1, 40, 2, 4, 2100, 128, 4, True),     # more work items than CTAs
+]
+
+
+@pytest.mark.parametrize("shape", MULTI_Q_SHAPES)
+def test_gqa_several_query_positions(flashd_lib, shape):
+    """A decode step over the last Nq positions: position iq sees keys 0 .. Nk-Nq+iq."""
+    B, Hkv, G, Nq, Nk, d, S, causal = shape
+    q, _, _ = synth.random_qkv(B, Hkv * G, Nq, 1, d, seed=800 + Nk)
+    _, k, v = synth.random_qkv(B, Hkv, 1, Nk, d, seed=801 + Nk)
+    sc = f32_scale(d)
+    q_index = [Nk - Nq + iq for iq in range(Nq)]
+    want, want_lse = oracle.attn_naive(q, k.repeat_interleave(G, dim=1), v.repeat_interleave(G, dim=1), sc, causal,
+                                       q_index=q_index, return_lse=True)
+    qc, kc, vc = q.cuda(), k.cuda(), v.cuda()
+    ws = flashd_lib.flashd_gqa_partial(qc, kc, vc, sc, S, causal=causal)
+    ok_status(flashd_lib)
+    assert tuple(ws.shape) == (B, Hkv * G, Nq, S, d + 1)
+    # a partial state is empty exactly when its split holds no visible key of that position
+    per = -(-Nk // S)
+    Lp = ws[..., d].cpu().numpy()
+    for iq in range(Nq):
+        lim = (Nk - Nq + iq + 1) if causal else Nk
+        for sp in range(S):
+            nonempty = sp * per < min(lim, Nk)
+            assert np.all(np.isfinite(Lp[:, :, iq, sp])) == nonempty and (nonempty or np.all(np.isneginf(Lp[:, :, iq, sp])))
+    got32, lse = flashd_lib.flashd_splitk_combine(ws, B, Hkv * G, Nq, d, S, out_dtype=torch.float32, return_lse=True)
+    e = np.abs(got32.double().cpu().numpy() - want)
+    assert e.max() <= 1e-2 and e.mean() <= 1e-3, (shape, e.max(), e.mean())
+    assert np.abs(lse.double().cpu().numpy() - want_lse).max() <= 1e-3
+    got = flashd_lib.flashd_attn_fwd_gqa(qc, kc, vc, sc, S, causal=causal)
+    ok_status(flashd_lib)
+    assert torch.equal(got, got32.to(torch.bfloat16))
+    check_bf16(got, want, shape)
+
+
 def test_gqa_matches_single_query_path_on_repeated_heads(flashd_lib):
     """Same function, two data paths: the grouped kernel on shared heads and the
     single-query split-K kernel on explicitly repeated heads agree to rounding."""
@@ -111,6 +155,17 @@ def test_gqa_rejects_bad_arguments(flashd_lib):
     with pytest.raises(ValueError):
         flashd_lib.flashd_attn_fwd_gqa(q[:, :3].contiguous().cuda(), torch.cat([k, k], 1).cuda(),
                                        torch.cat([v, v], 1).cuda(), 0.1, 1)
+    # G * Nq beyond the limit, and more causal positions than keys
+    q9, _, _ = synth.random_qkv(1, 3, 3, 1, 128, seed=2)
+    _, k1, v1 = synth.random_qkv(1, 1, 1, 64, 128, seed=3)
+    with pytest.raises(flashd_lib.FlashdError) as ei:
+        flashd_lib.flashd_attn_fwd_gqa(q9.cuda(), k1.cuda(), v1.cuda(), 0.1, 1)
+    assert ei.value.status == 3
+    q4, _, _ = synth.random_qkv(1, 1, 4, 1, 128, seed=2)
+    with pytest.raises(flashd_lib.FlashdError) as ei:
+        flashd_lib.flashd_attn_fwd_gqa(q4.cuda(), k1[:, :, :2].contiguous().cuda(), v1[:, :, :2].contiguous().cuda(), 0.1, 1,
+                                       causal=True)
+    assert ei.value.status == 2
 
 
 def test_gqa_long_context_sampled(flashd_lib):
