@@ -576,6 +576,36 @@ def main():
         "roofline": roof, "clocks": clocks, "gpu_launches": int(launches),
     }
 
+    if rank == 0 and world == 1 and not w.splitk:
+        # launch gaps: the same launches replayed from a CUDA graph (50 per replay)
+        try:
+            n_graph = 50
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                step(0)
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    for i in range(n_graph):
+                        step(i)
+            torch.cuda.current_stream().wait_stream(side)
+            for _ in range(3):
+                graph.replay()
+            torch.cuda.synchronize()
+            g0 = torch.cuda.Event(enable_timing=True); g1 = torch.cuda.Event(enable_timing=True)
+            reps = max(1, min(args.steps // n_graph, 40))
+            g0.record()
+            for _ in range(reps):
+                graph.replay()
+            g1.record()
+            torch.cuda.synchronize()
+            gms = g0.elapsed_time(g1) / (reps * n_graph)
+            line["cuda_graph"] = {"launches_per_replay": n_graph, "replays": reps, "ms_per_step": gms,
+                                  "value": w.flops / (gms * 1e-3) / 1e12, "unit": "TFLOP/s"}
+            del graph
+        except Exception as ex:  # the headline number stands on its own
+            line["cuda_graph"] = {"error": repr(ex)}
+
     if rank == 0 and not args.no_e2e:
         e2e = bench_e2e(fd, w, args.steps, args.warmup, torch)
         line["e2e"] = {"value": e2e["tflops"] * world, "unit": "TFLOP/s", "h2d_bytes_per_step": e2e["h2d"],
