@@ -28,9 +28,11 @@
 // tile plays the part of the sigmoid's division.
 //
 // Warp roles (16 warps): 0-3 weights of query tile 0, 4-7 weights of query tile 1,
-// 8-11 correction + epilogue, 12 MMA issue, 13 TMA loads, 14-15 idle.
-// Tensor memory (512 columns): S0 | S1 | O0 | O1; P_i overlays the first 64
-// columns of S_i as packed bf16 pairs.
+// 8-11 correction + epilogue, 12 MMA issue (whole warp in uniform control flow, one elected
+// lane issues), 13 TMA loads (one lane), 14-15 idle.
+// Tensor memory (512 columns), D = 128: S0 | S1 | O0 | O1, P_i overlays the first 64
+// columns of S_i as packed bf16 pairs and is handed to the P V product in two halves of 64
+// keys; D = 64: S0 | S1 | P0 | P1 | O0 | O1.
 // Every mbarrier wait is bounded; a wait that runs out records itself in the
 // device status word, raises the CTA's abort flag and the CTA drains and exits.
 #pragma once
@@ -50,7 +52,7 @@ struct PrefillCfg {
     static constexpr int kTileBytes = kPanels * kPanelBytes;     // one Q / K / V tile
     static constexpr int kStages = (D == 128) ? 4 : 6;           // K/V ring
     static constexpr int kThreads = 512;
-    static constexpr int kBarriers = 20 + 2 * kStages;
+    static constexpr int kBarriers = 22 + 2 * kStages;
     static constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + 3 * 2 * 128 * 4 + kBarriers * 8 + 64 + 1024;
     static constexpr uint32_t kTmemCols = 512;
     // At D = 64 tensor memory has room for P next to S (S0 S1 P0 P1 O0 O1 = 512 columns), so
@@ -192,6 +194,7 @@ struct PrefillParams {
     int n_work;         // BH * n_qpairs
 };
 
+
 // Wait bounded to about two seconds; also leaves when another thread of the CTA
 // has raised the abort flag.
 __device__ __forceinline__ bool pf_wait(uint64_t* bar, uint32_t parity, unsigned int which,
@@ -206,6 +209,25 @@ __device__ __forceinline__ bool pf_wait(uint64_t* bar, uint32_t parity, unsigned
     report_timeout(which, parity);
     *abort_flag = 1;
     return false;
+}
+
+// Non-blocking look at a barrier phase (a later pf_wait covers a miss).
+__device__ __forceinline__ uint32_t mbar_test(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok;
+}
+// One lane of a converged warp
+__device__ __forceinline__ uint32_t elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+    return pred;
 }
 
 template <int D>
@@ -237,8 +259,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     uint64_t* o_ready = bars + 14;      // [2]
     uint64_t* final_full = bars + 16;   // [2]
     uint64_t* s_free = bars + 18;       // [2]  S has been read into registers (lookahead 2 only)
-    uint64_t* kv_full = bars + 20;                 // [kStages]
-    uint64_t* kv_empty = bars + 20 + C::kStages;   // [kStages]
+    uint64_t* p_half = bars + 20;       // [2]  first 64 keys of P stored (lookahead 1 only)
+    uint64_t* kv_full = bars + 22;                 // [kStages]
+    uint64_t* kv_empty = bars + 22 + C::kStages;   // [kStages]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::kBarriers);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
@@ -254,6 +277,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             mbar_init(&alpha_full[i], 128);
             mbar_init(&final_full[i], 128);
             mbar_init(&s_free[i], 128);
+            mbar_init(&p_half[i], 128);
             mbar_init(&pv_done[i], 1);
             mbar_init(&o_ready[i], 128);
         }
@@ -323,115 +347,186 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
     } else if (warp == 12) {
         // ================================================================ MMA issue
+        // The whole warp runs the loop (uniform control flow, waits by all lanes); one elected
+        // lane issues the products and the commits.  The barriers the next batch of products
+        // will need are looked at between the products of the current batch, while the tensor
+        // pipe still has work queued, so that in the common case no wait sits between batches.
         reg_dec<96>();
-        if (lane == 0) {
+        {
+            const uint32_t leader = elect_one();
             constexpr uint32_t idesc_s = make_idesc(128, 128, 0);
             constexpr uint32_t idesc_o = make_idesc(128, D, 1);
             const uint32_t tS[2] = {tmem_base + C::kColS0, tmem_base + C::kColS1};
             const uint32_t tO[2] = {tmem_base + C::kColO0, tmem_base + C::kColO1};
             const uint32_t tP[2] = {tmem_base + C::kColP0, tmem_base + C::kColP1};
             uint32_t kv_it = 0;
-            uint32_t n_p[2] = {0, 0}, n_or[2] = {0, 0}, n_qf[2] = {0, 0};
-            // descriptor words: Q and K tiles are K-major (8-row groups 1024 bytes apart),
-            // V tiles are MN-major (8-key groups 1024 bytes apart, 64-column panels
-            // kPanelBytes apart)
+            uint32_t n_ph0 = 0, n_ph1 = 0;
+            uint32_t n_p0 = 0, n_p1 = 0, n_or0 = 0, n_or1 = 0, n_qf0 = 0, n_qf1 = 0, n_sf0 = 0, n_sf1 = 0;
             constexpr uint32_t desc_hi = smem_desc_hi(1024);
             const uint32_t q_lo[2] = {smem_desc_lo(smem_u32(sQ), 16), smem_desc_lo(smem_u32(sQ + C::kTileBytes), 16)};
             const uint32_t k_lo0 = smem_desc_lo(smem_u32(sKV), 16);
             const uint32_t v_lo0 = smem_desc_lo(smem_u32(sKV), C::kPanelBytes);
-            // The issuing thread shares its scheduler with busy warps, so every instruction it
-            // needs between two products delays the tensor pipe.  The descriptors of the next
-            // products are therefore built while the thread would wait anyway (prep_*), and the
-            // products themselves are issued back to back from registers (fire_*).
             constexpr int KS = D / 16;
-            uint64_t qd0[KS], qd1[KS], kd[KS], vd[8];
-#pragma unroll
-            for (int ks = 0; ks < KS; ++ks) {
-                const uint32_t off = ((ks >> 2) * C::kPanelBytes + (ks & 3) * 32) >> 4;
-                qd0[ks] = desc64(q_lo[0] + off, desc_hi);
-                qd1[ks] = desc64(q_lo[1] + off, desc_hi);
-            }
-            auto prep_K = [&](int stage) {
+            constexpr int LA = C::kLookahead;
+            auto koff = [](int ks) -> uint32_t { return (uint32_t)(((ks >> 2) * C::kPanelBytes + (ks & 3) * 32) >> 4); };
+            // products of one batch; mid(ks) runs on all lanes after product ks
+            auto fire_S = [&](int i, int stage, auto&& mid) {
                 const uint32_t ka = k_lo0 + stage * (C::kTileBytes >> 4);
 #pragma unroll
-                for (int ks = 0; ks < KS; ++ks)
-                    kd[ks] = desc64(ka + (((ks >> 2) * C::kPanelBytes + (ks & 3) * 32) >> 4), desc_hi);
+                for (int ks = 0; ks < KS; ++ks) {
+                    if (leader) mma_ss64(tS[i], desc64(q_lo[i] + koff(ks), desc_hi), desc64(ka + koff(ks), desc_hi), idesc_s, ks > 0);
+                    __syncwarp();
+                    mid(ks * (8 / KS));
+                }
             };
-            auto fire_S = [&](int i) {
-#pragma unroll
-                for (int ks = 0; ks < KS; ++ks) mma_ss64(tS[i], i == 0 ? qd0[ks] : qd1[ks], kd[ks], idesc_s, ks > 0);
-            };
-            auto prep_V = [&](int stage) {
+            auto fire_PV_part = [&](int i, int stage, bool first, int ks0) {
                 const uint32_t va = v_lo0 + stage * (C::kTileBytes >> 4);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) vd[ks] = desc64(va + ks * (2048 >> 4), desc_hi);   // 16 keys = two 1024-byte atoms
+                for (int ks = ks0; ks < ks0 + 4; ++ks) {
+                    if (leader) mma_ts64(tO[i], tP[i] + ks * 8, desc64(va + ks * (2048 >> 4), desc_hi), idesc_o, (!first) || ks > 0);
+                    __syncwarp();
+                }
             };
-            auto fire_PV = [&](int i, bool first) {
+            auto fire_PV = [&](int i, int stage, bool first, auto&& mid) {
+                const uint32_t va = v_lo0 + stage * (C::kTileBytes >> 4);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) mma_ts64(tO[i], tP[i] + ks * 8, vd[ks], idesc_o, (!first) || ks > 0);
+                for (int ks = 0; ks < 8; ++ks) {
+                    if (leader) mma_ts64(tO[i], tP[i] + ks * 8, desc64(va + ks * (2048 >> 4), desc_hi), idesc_o, (!first) || ks > 0);
+                    __syncwarp();
+                    mid(ks);
+                }
             };
-            constexpr int LA = C::kLookahead;
-            uint32_t n_sf[2] = {0, 0};
+            auto commit = [&](uint64_t* bar) {
+                if (leader) tc_commit(bar);
+                __syncwarp();
+            };
             for (int nw = 0, w = work_index(0); w < prm.n_work; w = work_index(++nw)) {
                 const int qpair = prm.n_qpairs - 1 - w / prm.BH;
                 const int q0 = qpair * 256;
-                const int Ti[2] = {n_tiles(q0), n_tiles(q0 + 128)};
-                const int T = max(Ti[0], Ti[1]);
-                // ring positions of this work item: K_t at kv_it + 2t, V_t at kv_it + 2t + 1
+                const int T0 = n_tiles(q0), T1 = n_tiles(q0 + 128);
+                const int T = max(T0, T1);
                 auto stage_of = [&](uint32_t it) { return (int)(it % C::kStages); };
                 auto parity_of = [&](uint32_t it) { return (it / C::kStages) & 1u; };
-                // S_i(u): score product of key tile u for query tile i; with lookahead 2 the S
-                // region must have been read by the weights warps of step u-1 first
-                auto do_S = [&](int i, int u) -> bool {
-                    if (u == 0) {
-                        if (!pf_wait(&q_full[i], n_qf[i] & 1, kWaitQFull, abort_flag)) return false;
-                        ++n_qf[i];
-                    } else if (LA > 1) {
-                        if (!pf_wait(&s_free[i], n_sf[i] & 1, kWaitSFree, abort_flag)) return false;
-                        ++n_sf[i];
-                    }
-                    tc_fence_after();
-                    fire_S(i);
-                    tc_commit(&s_full[i]);
-                    if (u + 1 == Ti[i]) tc_commit(&q_empty[i]);
-                    return true;
-                };
+                // "known complete" flags of the next unconsumed phase of each barrier
+                uint32_t e_sf0 = 0, e_sf1 = 0, e_pf0 = 0, e_pf1 = 0, e_or0 = 0, e_or1 = 0, e_kvv = 0, e_kvk = 0;
+                auto none = [](int) {};
                 // prologue: S_i(0) .. S_i(LA-1)
                 for (int u = 0; u < LA && u < T; ++u) {
                     const uint32_t it_k = kv_it + 2 * u;
-                    prep_K(stage_of(it_k));
                     if (!pf_wait(&kv_full[stage_of(it_k)], parity_of(it_k), kWaitKVFull, abort_flag)) goto done;
-                    for (int i = 0; i < 2; ++i)
-                        if (u < Ti[i] && !do_S(i, u)) goto done;
-                    tc_commit(&kv_empty[stage_of(it_k)]);
+                    if (u < T0) {
+                        if (u == 0) { if (!pf_wait(&q_full[0], n_qf0 & 1, kWaitQFull, abort_flag)) goto done; ++n_qf0; }
+                        else { if (!pf_wait(&s_free[0], n_sf0 & 1, kWaitSFree, abort_flag)) goto done; ++n_sf0; }
+                        tc_fence_after();
+                        fire_S(0, stage_of(it_k), none);
+                        commit(&s_full[0]);
+                        if (u + 1 == T0) commit(&q_empty[0]);
+                    }
+                    if (u < T1) {
+                        if (u == 0) { if (!pf_wait(&q_full[1], n_qf1 & 1, kWaitQFull, abort_flag)) goto done; ++n_qf1; }
+                        else { if (!pf_wait(&s_free[1], n_sf1 & 1, kWaitSFree, abort_flag)) goto done; ++n_sf1; }
+                        tc_fence_after();
+                        fire_S(1, stage_of(it_k), none);
+                        commit(&s_full[1]);
+                        if (u + 1 == T1) commit(&q_empty[1]);
+                    }
+                    commit(&kv_empty[stage_of(it_k)]);
                 }
                 for (int t = 0; t < T; ++t) {
                     const uint32_t it_v = kv_it + 2 * t + 1;
                     const uint32_t it_kn = kv_it + 2 * (t + LA);
-                    prep_V(stage_of(it_v));
-                    if (t + LA < T) prep_K(stage_of(it_kn));
-                    if (!pf_wait(&kv_full[stage_of(it_v)], parity_of(it_v), kWaitKVFull, abort_flag)) goto done;
-                    bool kn_ready = false;
-                    for (int i = 0; i < 2; ++i) {
-                        if (t < Ti[i]) {
-                            if (!pf_wait(&p_full[i], n_p[i] & 1, kWaitPFull, abort_flag)) goto done;
-                            ++n_p[i];
-                            if (!pf_wait(&o_ready[i], n_or[i] & 1, kWaitOReady, abort_flag)) goto done;
-                            ++n_or[i];
-                            tc_fence_after();
-                            fire_PV(i, t == 0);
-                            tc_commit(&pv_done[i]);
-                        }
-                        if (t + LA < Ti[i]) {
-                            if (!kn_ready) {
-                                if (!pf_wait(&kv_full[stage_of(it_kn)], parity_of(it_kn), kWaitKVFull, abort_flag)) goto done;
-                                kn_ready = true;
-                            }
-                            if (!do_S(i, t + LA)) goto done;
-                        }
+                    const int st_v = stage_of(it_v), st_k = stage_of(it_kn);
+                    const bool pv0 = t < T0, pv1 = t < T1, s0 = t + LA < T0, s1 = t + LA < T1;
+                    const bool nxt0 = t + 1 < T0;      // PV_0(t+1) exists
+                    if (!e_kvv && !pf_wait(&kv_full[st_v], parity_of(it_v), kWaitKVFull, abort_flag)) goto done;
+                    e_kvv = 0;
+                    if (pv0 && LA == 1) {
+                        // P overlays S, so S_0(t+1) has to follow P V_0(t) and the chain per tile is
+                        // weights -> P V -> S -> weights: the first four products (keys 0-63) are
+                        // issued under the second half of the weights step
+                        if (!e_or0 && !pf_wait(&o_ready[0], n_or0 & 1, kWaitOReady, abort_flag)) goto done;
+                        if (!pf_wait(&p_half[0], n_ph0 & 1, kWaitPFull, abort_flag)) goto done;
+                        e_or0 = 0; ++n_or0; ++n_ph0;
+                        tc_fence_after();
+                        fire_PV_part(0, st_v, t == 0, 0);
+                        if (s0 || s1) e_kvk = mbar_test(&kv_full[st_k], parity_of(it_kn));
+                        if (!pf_wait(&p_full[0], n_p0 & 1, kWaitPFull, abort_flag)) goto done;
+                        e_pf0 = 0; ++n_p0;
+                        tc_fence_after();
+                        fire_PV_part(0, st_v, false, 4);
+                        commit(&pv_done[0]);
+                    } else if (pv0) {
+                        if (!e_pf0 && !pf_wait(&p_full[0], n_p0 & 1, kWaitPFull, abort_flag)) goto done;
+                        if (!e_or0 && !pf_wait(&o_ready[0], n_or0 & 1, kWaitOReady, abort_flag)) goto done;
+                        e_pf0 = 0; e_or0 = 0; ++n_p0; ++n_or0;
+                        tc_fence_after();
+                        fire_PV(0, st_v, t == 0, [&](int ks) {
+                            if (ks == 2 && (s0 || s1)) e_kvk = mbar_test(&kv_full[st_k], parity_of(it_kn));
+                            if (ks == 4 && s0 && LA > 1) e_sf0 = mbar_test(&s_free[0], n_sf0 & 1);
+                            if (ks == 4 && !s0 && pv1) e_pf1 = mbar_test(&p_full[1], n_p1 & 1);
+                            if (ks == 5 && !s0 && pv1) e_or1 = mbar_test(&o_ready[1], n_or1 & 1);
+                        });
+                        commit(&pv_done[0]);
                     }
-                    tc_commit(&kv_empty[stage_of(it_v)]);
-                    if (t + LA < T) tc_commit(&kv_empty[stage_of(it_kn)]);
+                    if (s0) {
+                        if (!e_kvk && !pf_wait(&kv_full[st_k], parity_of(it_kn), kWaitKVFull, abort_flag)) goto done;
+                        e_kvk = 1;      // stays known for S_1 of this step
+                        if (LA > 1) {
+                            if (!e_sf0 && !pf_wait(&s_free[0], n_sf0 & 1, kWaitSFree, abort_flag)) goto done;
+                            e_sf0 = 0; ++n_sf0;
+                        }
+                        tc_fence_after();
+                        fire_S(0, st_k, [&](int ks) {
+                            if (ks == 2 && pv1) e_pf1 = mbar_test(&p_full[1], n_p1 & 1);
+                            if (ks == 4 && pv1) e_or1 = mbar_test(&o_ready[1], n_or1 & 1);
+                        });
+                        commit(&s_full[0]);
+                        if (t + LA + 1 == T0) commit(&q_empty[0]);
+                    }
+                    if (pv1 && LA == 1) {
+                        if (!e_or1 && !pf_wait(&o_ready[1], n_or1 & 1, kWaitOReady, abort_flag)) goto done;
+                        if (!pf_wait(&p_half[1], n_ph1 & 1, kWaitPFull, abort_flag)) goto done;
+                        e_or1 = 0; ++n_or1; ++n_ph1;
+                        tc_fence_after();
+                        fire_PV_part(1, st_v, t == 0, 0);
+                        if (s1 && !e_kvk) e_kvk = mbar_test(&kv_full[st_k], parity_of(it_kn));
+                        if (!pf_wait(&p_full[1], n_p1 & 1, kWaitPFull, abort_flag)) goto done;
+                        e_pf1 = 0; ++n_p1;
+                        tc_fence_after();
+                        fire_PV_part(1, st_v, false, 4);
+                        commit(&pv_done[1]);
+                    } else if (pv1) {
+                        if (!e_pf1 && !pf_wait(&p_full[1], n_p1 & 1, kWaitPFull, abort_flag)) goto done;
+                        if (!e_or1 && !pf_wait(&o_ready[1], n_or1 & 1, kWaitOReady, abort_flag)) goto done;
+                        e_pf1 = 0; e_or1 = 0; ++n_p1; ++n_or1;
+                        tc_fence_after();
+                        fire_PV(1, st_v, t == 0, [&](int ks) {
+                            if (ks == 2 && s1 && !e_kvk) e_kvk = mbar_test(&kv_full[st_k], parity_of(it_kn));
+                            if (ks == 4 && s1 && LA > 1) e_sf1 = mbar_test(&s_free[1], n_sf1 & 1);
+                            if (ks == 4 && !s1 && t + 1 < T) e_kvv = mbar_test(&kv_full[stage_of(it_v + 2)], parity_of(it_v + 2));
+                            if (ks == 5 && !s1 && nxt0) e_pf0 = mbar_test(&p_full[0], n_p0 & 1);
+                            if (ks == 6 && !s1 && nxt0) e_or0 = mbar_test(&o_ready[0], n_or0 & 1);
+                        });
+                        commit(&pv_done[1]);
+                    }
+                    if (s1) {
+                        if (!e_kvk && !pf_wait(&kv_full[st_k], parity_of(it_kn), kWaitKVFull, abort_flag)) goto done;
+                        if (LA > 1) {
+                            if (!e_sf1 && !pf_wait(&s_free[1], n_sf1 & 1, kWaitSFree, abort_flag)) goto done;
+                            e_sf1 = 0; ++n_sf1;
+                        }
+                        tc_fence_after();
+                        fire_S(1, st_k, [&](int ks) {
+                            if (ks == 0 && t + 1 < T) e_kvv = mbar_test(&kv_full[stage_of(it_v + 2)], parity_of(it_v + 2));
+                            if (ks == 2 && nxt0) e_pf0 = mbar_test(&p_full[0], n_p0 & 1);
+                            if (ks == 4 && nxt0) e_or0 = mbar_test(&o_ready[0], n_or0 & 1);
+                        });
+                        commit(&s_full[1]);
+                        if (t + LA + 1 == T1) commit(&q_empty[1]);
+                    }
+                    e_kvk = 0;
+                    commit(&kv_empty[st_v]);
+                    if (t + LA < T) commit(&kv_empty[st_k]);
                 }
                 kv_it += 2 * T;
             }
@@ -513,6 +608,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     uint32_t pk[32];
 #pragma unroll
                     for (int j = 0; j < 64; j += 4) {
+                        if (C::kLookahead == 1 && h == 1 && j == 32) {
+                            // the first 64 weights are in tensor memory: their product may start
+                            tc_wait_st();
+                            tc_fence_before();
+                            mbar_arrive(&p_half[i]);
+                        }
                         float x0, x1, x2, x3;
                         unpack2(fma2(pack2(s[64 * h + j], s[64 * h + j + 1]), c2, nref2), x0, x1);
                         unpack2(fma2(pack2(s[64 * h + j + 2], s[64 * h + j + 3]), c2, nref2), x2, x3);
