@@ -610,7 +610,7 @@ def main():
         e2e = bench_e2e(fd, w, args.steps, args.warmup, torch)
         line["e2e"] = {"value": e2e["tflops"] * world, "unit": "TFLOP/s", "h2d_bytes_per_step": e2e["h2d"],
                        "d2h_bytes_per_step": e2e["d2h"], "ms_per_step": e2e["ms_per_step"], "workload": e2e["workload"],
-                       "note": "flashd_attn_fwd_host: pinned host q,k,v -> device, kernel, o -> host, every step"}
+                       "note": "flashd_attn_fwd_host: pinned host q,k,v -> device, kernel, o -> host, every step (chunks of heads pipelined on three streams inside the call)"}
     if world > 1:
         # replicas: every rank does the same end-to-end work; report rank 0's rate times the replica count
         dist.barrier()

@@ -287,11 +287,16 @@ int flashd_skip_stats(const void* q, const void* k, unsigned long long* counts, 
 /* ------------------------------------------------------------------------
  * End-to-end call on HOST buffers: q, k, v, o are host pointers (pinned
  * memory gives asynchronous copies).  The call allocates device buffers from
- * the stream-ordered pool of the current device, copies q, k, v in, runs the
- * forward selected by `path`, copies o back, frees the buffers and
- * SYNCHRONISES `stream` before returning.
+ * the stream-ordered pool of the current device, cuts the batch into chunks
+ * of whole heads (about 12 MB of input each, at most 8) and pipelines them:
+ * chunk c+1 is copied in while chunk c runs the forward selected by `path`
+ * and chunk c-1 is copied out, on two helper streams of the library that
+ * start after the work already queued on `stream` and are joined back into
+ * it.  It frees the buffers and SYNCHRONISES `stream` before returning.
+ * Calls on the same device are serialised by a lock (they share the helper
+ * streams).  Not for use under stream capture.
  * path 0: flashd_attn_fwd (bf16)   path 1: flashd_attn_fwd_f32
- * path 2: flashd_attn_fwd_splitk (bf16, library's split count)            */
+ * path 2: flashd_attn_fwd_splitk (bf16, library's split count per chunk)   */
 int flashd_attn_fwd_host(const void* q, const void* k, const void* v, void* o,
                          int path, int B, int H, int Nq, int Nk, int d, float scale,
                          int causal, void* stream);

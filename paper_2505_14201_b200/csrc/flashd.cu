@@ -4,6 +4,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstdint>
@@ -259,6 +260,31 @@ int check_splits(int Nk, int num_splits) {
 }  // namespace
 
 // ============================================================================ C ABI
+// Per-device helper streams and events of the host entry point (created on first use).
+namespace {
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_out = nullptr;
+    cudaEvent_t ev_in[16] = {nullptr}, ev_k[16] = {nullptr};
+};
+HostPipe g_pipe[64];
+std::mutex g_pipe_mutex;
+
+bool host_pipe_init(HostPipe& hp) {
+    if (hp.ready) return true;
+    bool ok = cudaStreamCreateWithFlags(&hp.s_in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&hp.s_out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.ev_start, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.ev_out, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; ok && i < 16; ++i)
+        ok = cudaEventCreateWithFlags(&hp.ev_in[i], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&hp.ev_k[i], cudaEventDisableTiming) == cudaSuccess;
+    hp.ready = ok;
+    return ok;
+}
+}  // namespace
+
 extern "C" {
 
 int flashd_version(void) { return 100; }
@@ -534,21 +560,19 @@ int flashd_attn_fwd_host(const void* q, const void* k, const void* v, void* o, i
     if (B <= 0 || H <= 0 || Nq <= 0 || Nk <= 0 || d <= 0 || !std::isfinite(scale)) return FLASHD_ERR_SHAPE;
     if (path < 0 || path > 2) return FLASHD_ERR_UNSUPPORTED;
     if (path == 2 && causal) return FLASHD_ERR_UNSUPPORTED;
+    if ((long long)B * H > 0x7fffffffLL / 2) return FLASHD_ERR_SHAPE;
     const size_t esz = (path == 1) ? 4 : 2;
-    const size_t qb = (size_t)B * H * Nq * d * esz, kb = (size_t)B * H * Nk * d * esz;
+    const int BH = B * H;
+    const size_t q_head = (size_t)Nq * d * esz, k_head = (size_t)Nk * d * esz;   // bytes of one head
+    const size_t qb = q_head * BH, kb = k_head * BH;
     cudaStream_t s = as_stream(stream);
-    int splits = 0;
-    size_t wsb = 0;
-    if (path == 2) {
-        splits = flashd_splitk_num_splits(B, H, Nq, Nk, d);
-        wsb = flashd_splitk_workspace_bytes(B, H, Nq, d, splits);
-    }
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FLASHD_ERR_CUDA;
     // keep freed staging buffers in the device's default pool instead of returning them to
     // the driver at every synchronisation (set once per device)
     {
         static bool pool_set[64] = {false};
-        int dev = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64 && !pool_set[dev]) {
+        if (!pool_set[dev]) {
             cudaMemPool_t pool;
             if (cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess) {
                 unsigned long long keep = ~0ull;
@@ -557,21 +581,60 @@ int flashd_attn_fwd_host(const void* q, const void* k, const void* v, void* o, i
             pool_set[dev] = true;
         }
     }
-    void *dq = nullptr, *dk = nullptr, *dv = nullptr, *dout = nullptr, *dws = nullptr;
-    int st = FLASHD_OK;
-    bool ok = cudaMallocAsync(&dq, qb, s) == cudaSuccess && cudaMallocAsync(&dk, kb, s) == cudaSuccess &&
-              cudaMallocAsync(&dv, kb, s) == cudaSuccess && cudaMallocAsync(&dout, qb, s) == cudaSuccess &&
-              (wsb == 0 || cudaMallocAsync(&dws, wsb, s) == cudaSuccess);
-    ok = ok && cudaMemcpyAsync(dq, q, qb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
-         cudaMemcpyAsync(dk, k, kb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
-         cudaMemcpyAsync(dv, v, kb, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    if (!ok) st = FLASHD_ERR_CUDA;
-    if (st == FLASHD_OK) {
-        if (path == 0) st = flashd_attn_fwd(dq, dk, dv, dout, B, H, Nq, Nk, d, scale, causal, stream);
-        else if (path == 1) st = flashd_attn_fwd_f32(dq, dk, dv, dout, B, H, Nq, Nk, d, scale, causal, stream);
-        else st = flashd_attn_fwd_splitk(dq, dk, dv, dout, dws, wsb, B, H, Nq, Nk, d, scale, splits, stream);
+    // Heads are independent, so the batch is cut into chunks of whole heads and the three
+    // legs are pipelined on three streams: chunk c+1 is copied in while chunk c is computed
+    // and chunk c-1 is copied out (the two copy directions use different copy engines).
+    // About 12 MB of input per chunk, at most 8 chunks: every chunk costs some tens of
+    // microseconds of copy set-up, so finer cuts lose more than they overlap.
+    int chunks = (int)std::min<size_t>(8, std::max<size_t>(1, (qb + 2 * kb) / (12u << 20)));
+    if (chunks > BH) chunks = BH;
+    const int heads_per = (BH + chunks - 1) / chunks;
+    chunks = (BH + heads_per - 1) / heads_per;
+    int splits = 0;
+    size_t wsb = 0;
+    if (path == 2) {
+        splits = flashd_splitk_num_splits(1, heads_per, Nq, Nk, d);
+        wsb = flashd_splitk_workspace_bytes(1, heads_per, Nq, d, splits);
     }
-    if (st == FLASHD_OK && cudaMemcpyAsync(o, dout, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) st = FLASHD_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);     // the helper streams and events are shared per device
+    HostPipe& hp = g_pipe[dev];
+    if (!host_pipe_init(hp)) return FLASHD_ERR_CUDA;
+    char *dq = nullptr, *dk = nullptr, *dv = nullptr, *dout = nullptr;
+    void* dws = nullptr;
+    int st = FLASHD_OK;
+    bool ok = cudaMallocAsync((void**)&dq, qb, s) == cudaSuccess && cudaMallocAsync((void**)&dk, kb, s) == cudaSuccess &&
+              cudaMallocAsync((void**)&dv, kb, s) == cudaSuccess && cudaMallocAsync((void**)&dout, qb, s) == cudaSuccess &&
+              (wsb == 0 || cudaMallocAsync(&dws, wsb, s) == cudaSuccess);
+    // the helper streams start after everything already queued on `stream` (and the allocations)
+    ok = ok && cudaEventRecord(hp.ev_start, s) == cudaSuccess &&
+         cudaStreamWaitEvent(hp.s_in, hp.ev_start, 0) == cudaSuccess &&
+         cudaStreamWaitEvent(hp.s_out, hp.ev_start, 0) == cudaSuccess;
+    if (!ok) st = FLASHD_ERR_CUDA;
+    for (int c = 0; c < chunks && st == FLASHD_OK; ++c) {
+        const int h0 = c * heads_per;
+        const int nh = std::min(heads_per, BH - h0);
+        const size_t qo = q_head * h0, ko = k_head * h0;
+        ok = cudaMemcpyAsync(dq + qo, static_cast<const char*>(q) + qo, q_head * nh, cudaMemcpyHostToDevice, hp.s_in) == cudaSuccess &&
+             cudaMemcpyAsync(dk + ko, static_cast<const char*>(k) + ko, k_head * nh, cudaMemcpyHostToDevice, hp.s_in) == cudaSuccess &&
+             cudaMemcpyAsync(dv + ko, static_cast<const char*>(v) + ko, k_head * nh, cudaMemcpyHostToDevice, hp.s_in) == cudaSuccess &&
+             cudaEventRecord(hp.ev_in[c], hp.s_in) == cudaSuccess && cudaStreamWaitEvent(s, hp.ev_in[c], 0) == cudaSuccess;
+        if (!ok) { st = FLASHD_ERR_CUDA; break; }
+        if (path == 0) st = flashd_attn_fwd(dq + qo, dk + ko, dv + ko, dout + qo, 1, nh, Nq, Nk, d, scale, causal, stream);
+        else if (path == 1) st = flashd_attn_fwd_f32(dq + qo, dk + ko, dv + ko, dout + qo, 1, nh, Nq, Nk, d, scale, causal, stream);
+        else st = flashd_attn_fwd_splitk(dq + qo, dk + ko, dv + ko, dout + qo, dws, wsb, 1, nh, Nq, Nk, d, scale,
+                                         nh == heads_per ? splits : 0, stream);
+        if (st != FLASHD_OK) break;
+        ok = cudaEventRecord(hp.ev_k[c], s) == cudaSuccess && cudaStreamWaitEvent(hp.s_out, hp.ev_k[c], 0) == cudaSuccess &&
+             cudaMemcpyAsync(static_cast<char*>(o) + qo, dout + qo, q_head * nh, cudaMemcpyDeviceToHost, hp.s_out) == cudaSuccess;
+        if (!ok) st = FLASHD_ERR_CUDA;
+    }
+    // `stream` rejoins the helper streams before the buffers go back to the pool
+    if (cudaEventRecord(hp.ev_out, hp.s_out) != cudaSuccess || cudaStreamWaitEvent(s, hp.ev_out, 0) != cudaSuccess ||
+        cudaEventRecord(hp.ev_start, hp.s_in) != cudaSuccess || cudaStreamWaitEvent(s, hp.ev_start, 0) != cudaSuccess) {
+        if (st == FLASHD_OK) st = FLASHD_ERR_CUDA;
+        cudaStreamSynchronize(hp.s_in);
+        cudaStreamSynchronize(hp.s_out);
+    }
     if (dq) cudaFreeAsync(dq, s);
     if (dk) cudaFreeAsync(dk, s);
     if (dv) cudaFreeAsync(dv, s);

@@ -365,3 +365,26 @@ def test_host_entry_point(flashd_lib):
     want = oracle.attn_naive(q, k, v, f32_scale(w.d))
     got = flashd_lib.flashd_attn_fwd_host(q.pin_memory(), k.pin_memory(), v.pin_memory(), f32_scale(w.d), False, path=1)
     assert np.abs(got.double().numpy() - want).max() <= F32_MAX
+
+
+def test_host_entry_point_pipelined_chunks(flashd_lib):
+    """Inputs large enough for the host call to cut the batch into several chunks of heads
+    (ragged last chunk): the result must be the one of the device-pointer call, and right."""
+    q, k, v = synth.random_qkv(3, 7, 4096, 4096, 64, seed=43)
+    sc = f32_scale(64)
+    dev = flashd_lib.flashd_attn_fwd(q.cuda(), k.cuda(), v.cuda(), sc, False)
+    for _ in range(2):      # twice: the helper streams and events are reused
+        got = flashd_lib.flashd_attn_fwd_host(q.pin_memory(), k.pin_memory(), v.pin_memory(), sc, False, path=0)
+        assert torch.equal(got.view(torch.int16), dev.cpu().view(torch.int16))
+    for (b, h) in [(0, 0), (1, 4), (2, 6)]:
+        want = oracle.attn_naive(q[b:b + 1, h:h + 1], k[b:b + 1, h:h + 1], v[b:b + 1, h:h + 1], sc, False)
+        check_bf16(got[b:b + 1, h:h + 1], want, (b, h))
+    ok_status(flashd_lib)
+    # split-K path, one head per chunk
+    q, k, v = synth.random_qkv(2, 3, 1, 65536, 128, seed=44)
+    sc = f32_scale(128)
+    got = flashd_lib.flashd_attn_fwd_host(q.pin_memory(), k.pin_memory(), v.pin_memory(), sc, False, path=2)
+    for (b, h) in [(0, 0), (1, 2)]:
+        want = oracle.attn_naive(q[b:b + 1, h:h + 1], k[b:b + 1, h:h + 1], v[b:b + 1, h:h + 1], sc, False)
+        check_bf16(got[b:b + 1, h:h + 1], want, (b, h))
+    ok_status(flashd_lib)
