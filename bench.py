@@ -447,6 +447,44 @@ def run_gqa(fd, synth, torch, device, peaks, steps, batch=0):
                      "keys_per_s": w4.B * w4.H * w4.Nk / (ms * 1e-3), "kv_gb": (k.numel() + v.numel()) / 1e9}
     del q, k, v, ws, o
     torch.cuda.empty_cache()
+    # config 4 over a paged pool: pages of 256 keys in shuffled order, sequence lengths mixed
+    # uniformly between a quarter and the whole of Nk (a serving batch in mid-flight)
+    page = 256
+    g = torch.Generator(device=device).manual_seed(w4.seed + 7)
+    lens = torch.randint(w4.Nk // 4, w4.Nk + 1, (w4.B,), generator=g, device=device, dtype=torch.int32)
+    max_pages = w4.Nk // page
+    per_seq = (lens + page - 1) // page
+    num_pages = int(per_seq.sum().item())
+    perm = torch.randperm(num_pages, generator=g, device=device).to(torch.int32)
+    table = torch.zeros((w4.B, max_pages), dtype=torch.int32, device=device)
+    off = 0
+    for b in range(w4.B):
+        n = int(per_seq[b].item())
+        table[b, :n] = perm[off:off + n]
+        off += n
+    q = torch.randn(w4.B, w4.H, 1, w4.d, generator=g, device=device).to(torch.bfloat16)
+    kp = torch.empty(num_pages, w4.H, page, w4.d, dtype=torch.bfloat16, device=device)
+    vp = torch.empty_like(kp)
+    step_pages = max(1, num_pages // 64)
+    for p0 in range(0, num_pages, step_pages):
+        n = min(step_pages, num_pages - p0)
+        kp[p0:p0 + n] = torch.randn(n, w4.H, page, w4.d, generator=g, device=device).to(torch.bfloat16)
+        vp[p0:p0 + n] = torch.randn(n, w4.H, page, w4.d, generator=g, device=device).to(torch.bfloat16)
+    S = fd.flashd_splitk_num_splits(w4.B, w4.H, 1, w4.Nk, w4.d)
+    ws = torch.empty((w4.B, w4.H, 1, S, w4.d + 1), dtype=torch.float32, device=device)
+    o = torch.empty_like(q)
+    ms = time_gpu(lambda i: fd.flashd_attn_fwd_splitk_paged(q, kp, vp, table, lens, sc, S, workspace=ws, o=o),
+                  steps, 3, torch) / steps
+    keys = int(lens.sum().item()) * w4.H
+    alg = keys * w4.d * 2 * 2 + (q.numel() + o.numel()) * 2
+    out["paged"] = {"B": w4.B, "H": w4.H, "d": w4.d, "page_size": page, "num_pages": num_pages, "num_splits": S,
+                    "seq_lens": f"uniform in [{w4.Nk // 4}, {w4.Nk}], mean {float(lens.float().mean().item()):.0f}",
+                    "ms_per_step": ms, "gbs": alg / (ms * 1e-3) / 1e9,
+                    "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                    "frac_hbm_nominal": alg / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+                    "keys_per_s": keys / (ms * 1e-3), "kv_gb": keys * w4.d * 4 / 1e9}
+    del q, kp, vp, ws, o
+    torch.cuda.empty_cache()
     st, detail = fd.flashd_last_device_status()
     if st != 0:
         raise SystemExit(f"device status {st} {detail}")

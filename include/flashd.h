@@ -173,6 +173,49 @@ int flashd_attn_fwd_splitk(const void* q, const void* k, const void* v, void* o,
                            int num_splits, void* stream);
 
 /* ------------------------------------------------------------------------
+ * Split-K forward over a PAGED K/V cache with one length per sequence
+ * (decode in a serving loop).  The function is the one of
+ * flashd_attn_fwd_splitk, sequence by sequence (the paper treats one query
+ * over one key sequence, Sec. II-A; where the keys are stored and that
+ * sequences differ in length is outside it); only the addressing differs.
+ *
+ * k_pages, v_pages : [num_pages, H, page_size, d] bf16, contiguous, 16-byte
+ *                    aligned: the pool.  page_size must be a multiple of the
+ *                    kernel's ring stage (64 keys at d = 128, 128 at d = 64).
+ * block_table      : [B, max_pages] int32, DEVICE memory; entry (b, p) is the
+ *                    pool index of the page holding keys p*page_size ...
+ *                    (p+1)*page_size - 1 of sequence b.  Entries beyond the
+ *                    sequence's last page are not read.
+ * seq_lens         : [B] int32, DEVICE memory; keys of sequence b, in
+ *                    [0, max_pages*page_size].  A sequence of length 0 gives
+ *                    o = 0.
+ * q, o             : [B,H,Nq,d] bf16; every query row of sequence b sees all
+ *                    seq_lens[b] keys (non-causal).
+ * Each sequence's keys are cut into num_splits ranges of
+ * ceil(seq_lens[b] / num_splits) keys rounded up to whole ring stages (so
+ * short sequences leave late ranges empty); workspace and combine as for
+ * flashd_splitk_partial (flashd_splitk_workspace_bytes(B, H, Nq, d,
+ * num_splits)).  num_splits <= 0 in flashd_attn_fwd_splitk_paged selects
+ * flashd_splitk_num_splits(B, H, Nq, max_pages*page_size, d).
+ * The table and the lengths live on the device, so the host cannot check
+ * them: a length outside its range, or a page index outside
+ * [0, num_pages), is caught by the kernel, which then records
+ * FLASHD_ERR_SHAPE in the device status word (flashd_last_device_status),
+ * treats that sequence as empty or reads page 0 instead, and finishes;
+ * the output of that sequence is then meaningless.  No out-of-pool read is
+ * made.  Other errors as flashd_splitk_partial.                            */
+int flashd_splitk_partial_paged(const void* q, const void* k_pages, const void* v_pages,
+                                const int* block_table, const int* seq_lens,
+                                void* workspace, size_t workspace_bytes,
+                                int B, int H, int Nq, int max_pages, int page_size, int num_pages,
+                                int d, float scale, int num_splits, void* stream);
+int flashd_attn_fwd_splitk_paged(const void* q, const void* k_pages, const void* v_pages, void* o,
+                                 const int* block_table, const int* seq_lens,
+                                 void* workspace, size_t workspace_bytes,
+                                 int B, int H, int Nq, int max_pages, int page_size, int num_pages,
+                                 int d, float scale, int num_splits, void* stream);
+
+/* ------------------------------------------------------------------------
  * Split-K forward with K and V stored as FP8-E4M3 (the second number format of
  * the paper's evaluation, Sec. V-A).  q and o stay bf16; k, v : [B,H,Nk,d] of
  * one-byte E4M3 values (4 exponent bits, bias 7, 3 mantissa bits, no

@@ -20,6 +20,7 @@ EXPORTED_SYMBOLS = (
     "flashd_splitk_combine", "flashd_attn_fwd_splitk", "flashd_attn_fwd_splitk_static",
     "flashd_gqa_num_splits", "flashd_gqa_partial", "flashd_attn_fwd_gqa", "flashd_attn_fwd_pwl",
     "flashd_splitk_partial_fp8kv", "flashd_attn_fwd_splitk_fp8kv",
+    "flashd_splitk_partial_paged", "flashd_attn_fwd_splitk_paged",
     "flashd_attn_fwd_host", "flashd_skip_stats", "flashd_last_device_status", "flashd_status_string", "flashd_version", "flashd_launch_count",
 )
 
@@ -61,6 +62,8 @@ def lib() -> ctypes.CDLL:
             L.flashd_splitk_partial.argtypes = [vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_splitk_combine.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, vp]
             L.flashd_attn_fwd_splitk.argtypes = [vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
+            L.flashd_splitk_partial_paged.argtypes = [vp, vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, ci, ci, cf, ci, vp]
+            L.flashd_attn_fwd_splitk_paged.argtypes = [vp, vp, vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, ci, ci, cf, ci, vp]
             fp = ctypes.POINTER(ctypes.c_float)
             L.flashd_attn_fwd_pwl.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, ci,
                                               ci, fp, fp, ci, fp, fp, cf, cf, ci, vp]
@@ -265,6 +268,54 @@ def flashd_attn_fwd_splitk(q, k, v, scale, num_splits=0, workspace=None, o=None,
     _check(lib().flashd_attn_fwd_splitk(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(workspace),
                                         workspace.numel() * workspace.element_size(), B, H, Nq, Nk, d,
                                         float(scale), int(num_splits), _stream_ptr(stream)), "flashd_attn_fwd_splitk")
+    return o
+
+
+def _paged_dims(q, k_pages, v_pages, block_table, seq_lens):
+    import torch
+    for t in (q, k_pages, v_pages, block_table, seq_lens):
+        if not t.is_contiguous():
+            raise ValueError("paged split-K: all tensors must be contiguous")
+    if q.dim() != 4 or k_pages.dim() != 4 or tuple(v_pages.shape) != tuple(k_pages.shape):
+        raise ValueError("paged split-K: q [B,H,Nq,d], k_pages / v_pages [num_pages,H,page_size,d]")
+    B, H, Nq, d = q.shape
+    num_pages, Hk, page_size, dk = k_pages.shape
+    if Hk != H or dk != d or block_table.dim() != 2 or block_table.shape[0] != B or tuple(seq_lens.shape) != (B,):
+        raise ValueError("paged split-K: shapes do not match")
+    if block_table.dtype != torch.int32 or seq_lens.dtype != torch.int32:
+        raise ValueError("paged split-K: block_table and seq_lens must be int32")
+    return B, H, Nq, d, num_pages, page_size, block_table.shape[1]
+
+
+def flashd_splitk_partial_paged(q, k_pages, v_pages, block_table, seq_lens, scale, num_splits, workspace=None,
+                                stream=None):
+    """Partial states ``[B,H,Nq,num_splits,d+1]`` fp32 of the split-K forward over a paged K/V pool."""
+    import torch
+    B, H, Nq, d, num_pages, page_size, max_pages = _paged_dims(q, k_pages, v_pages, block_table, seq_lens)
+    if workspace is None:
+        workspace = torch.empty((B, H, Nq, num_splits, d + 1), dtype=torch.float32, device=q.device)
+    _check(lib().flashd_splitk_partial_paged(_ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(block_table), _ptr(seq_lens),
+                                             _ptr(workspace), workspace.numel() * workspace.element_size(), B, H, Nq,
+                                             max_pages, page_size, num_pages, d, float(scale), int(num_splits),
+                                             _stream_ptr(stream)), "flashd_splitk_partial_paged")
+    return workspace
+
+
+def flashd_attn_fwd_splitk_paged(q, k_pages, v_pages, block_table, seq_lens, scale, num_splits=0, workspace=None,
+                                 o=None, stream=None):
+    """Split-K forward over a paged K/V pool with one length per sequence (partial + combine)."""
+    import torch
+    B, H, Nq, d, num_pages, page_size, max_pages = _paged_dims(q, k_pages, v_pages, block_table, seq_lens)
+    S = num_splits if num_splits > 0 else flashd_splitk_num_splits(B, H, Nq, max_pages * page_size, d)
+    if workspace is None:
+        workspace = torch.empty((B, H, Nq, max(S, 1), d + 1), dtype=torch.float32, device=q.device)
+    if o is None:
+        o = torch.empty_like(q)
+    _check(lib().flashd_attn_fwd_splitk_paged(_ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(o), _ptr(block_table),
+                                              _ptr(seq_lens), _ptr(workspace),
+                                              workspace.numel() * workspace.element_size(), B, H, Nq, max_pages,
+                                              page_size, num_pages, d, float(scale), int(num_splits),
+                                              _stream_ptr(stream)), "flashd_attn_fwd_splitk_paged")
     return o
 
 

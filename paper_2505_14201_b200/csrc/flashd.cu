@@ -180,15 +180,15 @@ bool fill_table(int n, const float* x, const float* y, int* n_out, float* xs, fl
     return true;
 }
 
-template <int D, int KVB = 2>
+template <int D, int KVB = 2, bool PAGED = false>
 int launch_partial(const void* q, const void* k, const void* v, void* ws, long long rows, int Nq, int Nk,
-                   float scale, int num_splits, cudaStream_t stream) {
+                   float scale, int num_splits, cudaStream_t stream, const PagedKV& pg = PagedKV{}) {
     using C = DecodeCfg<D, KVB>;
     static bool attr_set[64] = {false};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FLASHD_ERR_CUDA;
     if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(splitk_partial_kernel<D, KVB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(splitk_partial_kernel<D, KVB, PAGED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  C::kSmemBytes) != cudaSuccess)
             return FLASHD_ERR_CUDA;
         attr_set[dev] = true;
@@ -197,9 +197,9 @@ int launch_partial(const void* q, const void* k, const void* v, void* ws, long l
     if (sms <= 0) return FLASHD_ERR_CUDA;
     const long long items = rows * num_splits;
     const int grid = (int)(items < sms ? items : sms);
-    splitk_partial_kernel<D, KVB><<<grid, C::kThreads, C::kSmemBytes, stream>>>(
+    splitk_partial_kernel<D, KVB, PAGED><<<grid, C::kThreads, C::kSmemBytes, stream>>>(
         static_cast<const __nv_bfloat16*>(q), static_cast<const unsigned char*>(k),
-        static_cast<const unsigned char*>(v), static_cast<float*>(ws), rows, Nq, Nk, scale * kLog2e, num_splits);
+        static_cast<const unsigned char*>(v), static_cast<float*>(ws), rows, Nq, Nk, scale * kLog2e, num_splits, pg);
     return after_launch();
 }
 
@@ -452,6 +452,52 @@ int flashd_attn_fwd_splitk_fp8kv(const void* q, const void* k, const void* v, vo
     if (num_splits <= 0) num_splits = flashd_splitk_num_splits(B, H, Nq, Nk, d);
     const int st = flashd_splitk_partial_fp8kv(q, k, v, workspace, workspace_bytes, B, H, Nq, Nk, d, scale,
                                                num_splits, stream);
+    if (st != FLASHD_OK) return st;
+    return flashd_splitk_combine(workspace, o, nullptr, B, H, Nq, d, num_splits, FLASHD_BF16, stream);
+}
+
+int flashd_splitk_partial_paged(const void* q, const void* k_pages, const void* v_pages, const int* block_table,
+                                const int* seq_lens, void* workspace, size_t workspace_bytes, int B, int H, int Nq,
+                                int max_pages, int page_size, int num_pages, int d, float scale, int num_splits,
+                                void* stream) {
+    if (!q || !k_pages || !v_pages || !block_table || !seq_lens || !workspace) return FLASHD_ERR_NULL;
+    if (B <= 0 || H <= 0 || Nq <= 0 || max_pages <= 0 || page_size <= 0 || num_pages <= 0 || d <= 0 ||
+        !std::isfinite(scale))
+        return FLASHD_ERR_SHAPE;
+    if ((long long)B * H > 0x7fffffffLL / 2 || (long long)max_pages * page_size > 0x7fffffffLL) return FLASHD_ERR_SHAPE;
+    if (!aligned16(q) || !aligned16(k_pages) || !aligned16(v_pages) || !aligned16(workspace) ||
+        (reinterpret_cast<uintptr_t>(block_table) & 3u) || (reinterpret_cast<uintptr_t>(seq_lens) & 3u))
+        return FLASHD_ERR_ALIGN;
+    if (d != 128 && d != 64) return FLASHD_ERR_UNSUPPORTED;
+    const int chunk = (d == 128) ? DecodeCfg<128>::kChunk : DecodeCfg<64>::kChunk;
+    if (page_size % chunk != 0) return FLASHD_ERR_UNSUPPORTED;     // a ring stage must not straddle pages
+    if (num_splits < 1 || num_splits > FLASHD_MAX_SPLITS) return FLASHD_ERR_WORKSPACE;
+    if (workspace_bytes < flashd_splitk_workspace_bytes(B, H, Nq, d, num_splits)) return FLASHD_ERR_WORKSPACE;
+    const long long rows = (long long)B * H * Nq;
+    if (rows > 0x7fffffffLL) return FLASHD_ERR_SHAPE;
+    PagedKV pg;
+    pg.block_table = block_table;
+    pg.seq_lens = seq_lens;
+    pg.max_pages = max_pages;
+    pg.page_size = page_size;
+    pg.num_pages = num_pages;
+    pg.H = H;
+    if (d == 128)
+        return launch_partial<128, 2, true>(q, k_pages, v_pages, workspace, rows, Nq, 0, scale, num_splits, as_stream(stream), pg);
+    return launch_partial<64, 2, true>(q, k_pages, v_pages, workspace, rows, Nq, 0, scale, num_splits, as_stream(stream), pg);
+}
+
+int flashd_attn_fwd_splitk_paged(const void* q, const void* k_pages, const void* v_pages, void* o,
+                                 const int* block_table, const int* seq_lens, void* workspace,
+                                 size_t workspace_bytes, int B, int H, int Nq, int max_pages, int page_size,
+                                 int num_pages, int d, float scale, int num_splits, void* stream) {
+    if (!o) return FLASHD_ERR_NULL;
+    if (!aligned16(o)) return FLASHD_ERR_ALIGN;
+    if (num_splits <= 0 && B > 0 && H > 0 && Nq > 0 && max_pages > 0 && page_size > 0 &&
+        (long long)max_pages * page_size <= 0x7fffffffLL)
+        num_splits = flashd_splitk_num_splits(B, H, Nq, max_pages * page_size, d);
+    const int st = flashd_splitk_partial_paged(q, k_pages, v_pages, block_table, seq_lens, workspace, workspace_bytes,
+                                               B, H, Nq, max_pages, page_size, num_pages, d, scale, num_splits, stream);
     if (st != FLASHD_OK) return st;
     return flashd_splitk_combine(workspace, o, nullptr, B, H, Nq, d, num_splits, FLASHD_BF16, stream);
 }

@@ -14,6 +14,12 @@
 //     o <- o + (o_p - o) W,  L <- L_p - ln W.
 // L is kept in log2 units inside the kernels and written in natural log.
 //
+// Paged variant (PAGED = true): K and V live in a pool of fixed-size pages
+// [num_pages, H, page_size, D]; sequence b owns the pages block_table[b][0..] in order and
+// has its own length seq_lens[b].  The split ranges are then cut per sequence, in multiples
+// of a ring stage, so that a stage never straddles two pages.  The function computed per
+// sequence is the one of the contiguous kernel.
+//
 // K and V are stored either as bf16 (KVB = 2 bytes per element) or as FP8-E4M3
 // (KVB = 1; the second number format of Sec. V-A).  E4M3 rows are half as long, so
 // the same bytes per ring stage hold twice the keys; every element is widened
@@ -42,6 +48,18 @@ struct DecodeCfg {
     static constexpr int kMergeFloats = kGroups * (D + 1);
     static constexpr int kSmemBytes = kStages * kStageBytes + kMergeFloats * 4 + 256;
 };
+
+// Page pool description of the paged variant (all pointers are device pointers).
+struct PagedKV {
+    const int* block_table;   // [B, max_pages] page index of the p-th page of sequence b
+    const int* seq_lens;      // [B] keys of sequence b
+    int max_pages;            // row length of block_table
+    int page_size;            // keys per page, a multiple of DecodeCfg::kChunk
+    int num_pages;            // pages in the pool
+    int H;                    // heads (pool layout [num_pages, H, page_size, D])
+};
+// detail code stored in the status word when a sequence length or page index is out of range
+enum { kBadPageTable = 0x1f0 };
 
 // which-wait codes reported on timeout
 enum { kWaitDecFull = 0x100, kWaitDecEmpty = 0x101, kWaitDecMergeReady = 0x102, kWaitDecMergeFree = 0x103 };
@@ -86,11 +104,23 @@ template <> __device__ __forceinline__ void widen_slice<1>(const uint4& raw, flo
     }
 }
 
-template <int D, int KVB>
+// keys [k0, k1) of split `split` of a sequence of Nk keys.  Contiguous K/V: ceil(Nk/S) keys per
+// split (per_split precomputed).  Paged: the same, rounded up to whole ring stages.
+template <int CHUNK, bool PAGED>
+__device__ __forceinline__ void split_range(int Nk, int num_splits, int per_split, int split, int& k0, int& k1) {
+    if (PAGED) {
+        const int ps = (Nk + num_splits - 1) / num_splits;
+        per_split = (ps + CHUNK - 1) / CHUNK * CHUNK;
+    }
+    k0 = min(split * per_split, Nk);
+    k1 = min(k0 + per_split, Nk);
+}
+
+template <int D, int KVB, bool PAGED = false>
 __global__ void __launch_bounds__(DecodeCfg<D, KVB>::kThreads, 1)
 splitk_partial_kernel(const __nv_bfloat16* __restrict__ q, const unsigned char* __restrict__ k,
                       const unsigned char* __restrict__ v, float* __restrict__ workspace,
-                      long long rows, int Nq, int Nk, float scale_log2e, int num_splits) {
+                      long long rows, int Nq, int Nk, float scale_log2e, int num_splits, const PagedKV pg) {
     using C = DecodeCfg<D, KVB>;
     constexpr int EL = C::kElems;
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -123,8 +153,24 @@ splitk_partial_kernel(const __nv_bfloat16* __restrict__ q, const unsigned char* 
             const long long row = item / num_splits;
             const int split = (int)(item - row * num_splits);
             const long long bh = row / Nq;
-            const int k0 = split * per_split;
-            const int k1 = min(k0 + per_split, Nk);
+            int seq_nk = Nk;
+            const int* pages = nullptr;
+            int head = 0;
+            if (PAGED) {
+                const int b = (int)(bh / pg.H);
+                head = (int)(bh - (long long)b * pg.H);
+                seq_nk = pg.seq_lens[b];
+                pages = pg.block_table + (long long)b * pg.max_pages;
+                if (seq_nk < 0 || seq_nk > pg.max_pages * pg.page_size) {
+                    // a length the table cannot hold: flag it and treat the sequence as empty
+                    if (atomicCAS(&g_status[0], 0u, (unsigned int)FLASHD_ERR_SHAPE) == 0u) {
+                        g_status[1] = blockIdx.x; g_status[2] = kBadPageTable; g_status[3] = (unsigned int)b;
+                    }
+                    seq_nk = 0;
+                }
+            }
+            int k0, k1;
+            split_range<C::kChunk, PAGED>(seq_nk, num_splits, per_split, split, k0, k1);
             const unsigned char* kb = k + (bh * Nk) * (long long)(D * KVB);
             const unsigned char* vb = v + (bh * Nk) * (long long)(D * KVB);
             for (int c0 = k0; c0 < k1; c0 += C::kChunk, ++it) {
@@ -134,9 +180,23 @@ splitk_partial_kernel(const __nv_bfloat16* __restrict__ q, const unsigned char* 
                 const int nk = min(C::kChunk, k1 - c0);
                 const uint32_t bytes = (uint32_t)nk * D * KVB;
                 unsigned char* dst = ring + stage * C::kStageBytes;
+                long long src = (long long)c0 * (D * KVB);
+                if (PAGED) {
+                    int page = pages[c0 / pg.page_size];
+                    if ((unsigned int)page >= (unsigned int)pg.num_pages) {
+                        // a page outside the pool: flag it and read page 0 so that the pipeline completes
+                        if (atomicCAS(&g_status[0], 0u, (unsigned int)FLASHD_ERR_SHAPE) == 0u) {
+                            g_status[1] = blockIdx.x; g_status[2] = kBadPageTable; g_status[3] = (unsigned int)page;
+                        }
+                        page = 0;
+                    }
+                    src = (((long long)page * pg.H + head) * pg.page_size + c0 % pg.page_size) * (long long)(D * KVB);
+                    kb = k;
+                    vb = v;
+                }
                 mbar_arrive_expect_tx(&full[stage], 2 * bytes);
-                bulk_load(dst, kb + (long long)c0 * (D * KVB), bytes, &full[stage]);
-                bulk_load(dst + C::kTileBytes, vb + (long long)c0 * (D * KVB), bytes, &full[stage]);
+                bulk_load(dst, kb + src, bytes, &full[stage]);
+                bulk_load(dst + C::kTileBytes, vb + src, bytes, &full[stage]);
             }
         }
         return;
@@ -150,8 +210,13 @@ splitk_partial_kernel(const __nv_bfloat16* __restrict__ q, const unsigned char* 
     for (long long item = blockIdx.x; item < n_items; item += gridDim.x, ++item_idx) {
         const long long row = item / num_splits;
         const int split = (int)(item - row * num_splits);
-        const int k0 = split * per_split;
-        const int k1 = min(k0 + per_split, Nk);
+        int seq_nk = Nk;
+        if (PAGED) {
+            seq_nk = pg.seq_lens[(row / Nq) / pg.H];
+            if (seq_nk < 0 || seq_nk > pg.max_pages * pg.page_size) seq_nk = 0;
+        }
+        int k0, k1;
+        split_range<C::kChunk, PAGED>(seq_nk, num_splits, per_split, split, k0, k1);
 
         float qf[EL];
 #pragma unroll

@@ -73,6 +73,16 @@ def test_validation_happens_before_any_launch(flashd_lib):
     assert part(a, a, a, a, ws_need, 1, 1, 1, 1024, 96, 0.1, 4, None) == 3
     assert L.flashd_splitk_combine(null, a, None, 1, 1, 1, 128, 4, 0, None) == 1
     assert L.flashd_splitk_combine(a, a, None, 1, 1, 1, 128, 0, 0, None) == 5
+    # paged split-K: (q, k_pages, v_pages, table, lens, ws, ws_bytes, B, H, Nq, max_pages, page_size, num_pages, d, scale, S)
+    pp = L.flashd_splitk_partial_paged
+    assert pp(a, a, a, null, a, a, ws_need, 1, 1, 1, 4, 64, 8, 128, 0.1, 4, None) == 1
+    assert pp(a, a, a, a, a, a, ws_need, 1, 1, 1, 4, 0, 8, 128, 0.1, 4, None) == 2
+    assert pp(a, a, a, a, a, a, ws_need, 1, 1, 1, 4, 96, 8, 128, 0.1, 4, None) == 3     # page not a multiple of the ring stage
+    assert pp(a, a, a, a, a, a, ws_need, 1, 1, 1, 4, 64, 8, 64, 0.1, 4, None) == 3      # d = 64 needs pages of 128 keys
+    assert pp(a, a, a, ctypes.c_void_p(a.value + 2), a, a, ws_need, 1, 1, 1, 4, 64, 8, 128, 0.1, 4, None) == 4
+    assert pp(a, a, a, a, a, a, ws_need - 1, 1, 1, 1, 4, 64, 8, 128, 0.1, 4, None) == 5
+    assert pp(a, a, a, a, a, a, ws_need, 1, 1, 1, 4, 64, 8, 128, 0.1, 65, None) == 5
+    assert L.flashd_attn_fwd_splitk_paged(a, a, a, null, a, a, a, ws_need, 1, 1, 1, 4, 64, 8, 128, 0.1, 4, None) == 1
     assert L.flashd_attn_fwd_host(a, a, a, a, 7, 1, 1, 8, 8, 64, 0.1, 0, None) == 3
     assert L.flashd_attn_fwd_host(a, a, a, a, 2, 1, 1, 8, 8, 64, 0.1, 1, None) == 3  # split-K is non-causal
     assert flashd_lib.launch_count() == n0
