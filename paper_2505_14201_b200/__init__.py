@@ -7,7 +7,7 @@ library or a CUDA device is missing.
 """
 from .binding import (  # noqa: F401
     FlashdError, lib, lib_path, status_string, version, launch_count,
-    flashd_attn_fwd, flashd_attn_fwd_ex, flashd_attn_fwd_f32, flashd_attn_fwd_perkey,
+    flashd_attn_fwd, flashd_attn_fwd_ex, flashd_attn_fwd_f32, flashd_attn_fwd_perkey, flashd_attn_fwd_fp8,
     flashd_splitk_workspace_bytes, flashd_splitk_num_splits, flashd_splitk_partial,
     flashd_splitk_combine, flashd_attn_fwd_splitk, flashd_attn_fwd_splitk_static, flashd_attn_fwd_host,
     flashd_gqa_num_splits, flashd_gqa_partial, flashd_attn_fwd_gqa, MAX_GROUP,

@@ -20,7 +20,7 @@ EXPORTED_SYMBOLS = (
     "flashd_splitk_combine", "flashd_attn_fwd_splitk", "flashd_attn_fwd_splitk_static",
     "flashd_gqa_num_splits", "flashd_gqa_partial", "flashd_attn_fwd_gqa", "flashd_attn_fwd_pwl",
     "flashd_splitk_partial_fp8kv", "flashd_attn_fwd_splitk_fp8kv",
-    "flashd_splitk_partial_paged", "flashd_attn_fwd_splitk_paged",
+    "flashd_splitk_partial_paged", "flashd_attn_fwd_splitk_paged", "flashd_attn_fwd_fp8",
     "flashd_attn_fwd_host", "flashd_skip_stats", "flashd_last_device_status", "flashd_status_string", "flashd_version", "flashd_launch_count",
 )
 
@@ -56,6 +56,7 @@ def lib() -> ctypes.CDLL:
             ex = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_attn_fwd_ex.argtypes = ex
             L.flashd_attn_fwd_perkey.argtypes = ex
+            L.flashd_attn_fwd_fp8.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_splitk_workspace_bytes.argtypes = [ci, ci, ci, ci, ci]
             L.flashd_splitk_workspace_bytes.restype = sz
             L.flashd_splitk_num_splits.argtypes = [ci, ci, ci, ci, ci]
@@ -158,6 +159,23 @@ def flashd_attn_fwd_ex(q, k, v, scale, causal=False, out_dtype=None, return_lse=
     _check(lib().flashd_attn_fwd_ex(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _dtype_code(q),
                                     _dtype_code(o), B, H, Nq, Nk, d, float(scale), int(bool(causal)),
                                     _stream_ptr(stream)), "flashd_attn_fwd_ex")
+    return (o, lse) if return_lse else o
+
+
+def flashd_attn_fwd_fp8(q, k, v, scale, causal=False, out_dtype=None, return_lse=False, o=None, stream=None):
+    """Tiled tensor-core forward with E4M3 operands (``torch.float8_e4m3fn`` q, k, v; d = 128);
+    output bf16 (default) or fp32."""
+    import torch
+    B, H, Nq, Nk, d = _dims(q, k, v)
+    for t in (q, k, v):
+        if t.dtype != torch.float8_e4m3fn:
+            raise ValueError("flashd_attn_fwd_fp8 takes torch.float8_e4m3fn tensors")
+    out_dtype = torch.bfloat16 if out_dtype is None else out_dtype
+    if o is None:
+        o = torch.empty(q.shape, dtype=out_dtype, device=q.device)
+    lse = torch.empty((B, H, Nq), dtype=torch.float32, device=q.device) if return_lse else None
+    _check(lib().flashd_attn_fwd_fp8(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _dtype_code(o), B, H, Nq, Nk, d,
+                                     float(scale), int(bool(causal)), _stream_ptr(stream)), "flashd_attn_fwd_fp8")
     return (o, lse) if return_lse else o
 
 

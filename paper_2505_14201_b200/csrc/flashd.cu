@@ -72,32 +72,33 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// [BH, N, D] bf16 tensor, box = 64 columns x 128 rows x 1 head, 128-byte swizzle,
-// rows outside [0, N) read as zero.
-bool make_map(CUtensorMap* map, const void* base, int BH, int N, int D) {
+// [BH, N, D] tensor of bf16 (eb = 2) or one-byte E4M3 (eb = 1) elements, box = 128 bytes of
+// columns x 128 rows x 1 head, 128-byte swizzle, rows outside [0, N) read as zero.
+bool make_map(CUtensorMap* map, const void* base, int BH, int N, int D, int eb = 2) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)N, (cuuint64_t)BH};
-    const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)N * D * 2};
-    const cuuint32_t box[3] = {64, 128, 1};
+    const cuuint64_t strides[2] = {(cuuint64_t)D * eb, (cuuint64_t)N * D * eb};
+    const cuuint32_t box[3] = {(cuuint32_t)(128 / eb), 128, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+    return fn(map, eb == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 3,
+              const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D>
+template <int D, int EB = 2>
 int launch_prefill(const void* q, const void* k, const void* v, void* o, float* lse, int out_f32, int BH, int Nq,
                    int Nk, float scale, int causal, cudaStream_t stream) {
-    using C = PrefillCfg<D>;
+    using C = PrefillCfg<D, EB>;
     CUtensorMap mq, mk, mv;
-    if (!make_map(&mq, q, BH, Nq, D) || !make_map(&mk, k, BH, Nk, D) || !make_map(&mv, v, BH, Nk, D))
+    if (!make_map(&mq, q, BH, Nq, D, EB) || !make_map(&mk, k, BH, Nk, D, EB) || !make_map(&mv, v, BH, Nk, D, EB))
         return FLASHD_ERR_CUDA;
     static bool attr_set[64] = {false};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FLASHD_ERR_CUDA;
     if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(prefill_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) !=
+        if (cudaFuncSetAttribute(prefill_kernel<D, EB>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) !=
             cudaSuccess)
             return FLASHD_ERR_CUDA;
         attr_set[dev] = true;
@@ -116,7 +117,7 @@ int launch_prefill(const void* q, const void* k, const void* v, void* o, float* 
     const int sms = sm_count();
     if (sms <= 0) return FLASHD_ERR_CUDA;
     const int grid = prm.n_work < sms ? prm.n_work : sms;
-    prefill_kernel<D><<<grid, C::kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, prm);
+    prefill_kernel<D, EB><<<grid, C::kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, prm);
     return after_launch();
 }
 
@@ -316,6 +317,17 @@ int flashd_attn_fwd_ex(const void* q, const void* k, const void* v, void* o, flo
     if (d == 128) return launch_prefill<128>(q, k, v, o, lse_out, out_dtype == FLASHD_F32, BH, Nq, Nk, scale, causal, as_stream(stream));
     if (d == 64) return launch_prefill<64>(q, k, v, o, lse_out, out_dtype == FLASHD_F32, BH, Nq, Nk, scale, causal, as_stream(stream));
     return FLASHD_ERR_UNSUPPORTED;
+}
+
+int flashd_attn_fwd_fp8(const void* q, const void* k, const void* v, void* o, float* lse_out, int out_dtype, int B,
+                        int H, int Nq, int Nk, int d, float scale, int causal, void* stream) {
+    const int st = check_common(q, k, v, o, B, H, Nq, Nk, d, scale);
+    if (st != FLASHD_OK) return st;
+    if (out_dtype != FLASHD_BF16 && out_dtype != FLASHD_F32) return FLASHD_ERR_UNSUPPORTED;
+    if (d != 128 || scale == 0.f) return FLASHD_ERR_UNSUPPORTED;
+    if (o == q || o == k || o == v) return FLASHD_ERR_SHAPE;
+    return launch_prefill<128, 1>(q, k, v, o, lse_out, out_dtype == FLASHD_F32, B * H, Nq, Nk, scale, causal,
+                                  as_stream(stream));
 }
 
 int flashd_attn_fwd(const void* q, const void* k, const void* v, void* o, int B, int H, int Nq, int Nk, int d,

@@ -43,11 +43,20 @@
 
 namespace flashd {
 
-template <int D>
+// EB = bytes per element of Q, K, V and P: 2 (bf16, tcgen05.mma kind::f16) or 1 (FP8-E4M3,
+// kind::f8f6f4; D = 128 only).  A product instruction covers 32 bytes of the contraction
+// dimension: 16 bf16 or 32 E4M3 elements.
+template <int D, int EB = 2>
 struct PrefillCfg {
+    static_assert(EB == 2 || (EB == 1 && D == 128), "E4M3 operands: D = 128 only");
     static constexpr int kBlockM = 128;
     static constexpr int kBlockN = 128;
-    static constexpr int kPanels = D / 64;                       // 64-column (128-byte) swizzle panels
+    static constexpr int kPanels = D * EB / 128;                 // 128-byte swizzle panels (64 bf16 / 128 E4M3 columns)
+    static constexpr int kPanelCols = 128 / EB;
+    static constexpr int kStepsS = D * EB / 32;                  // product instructions of S = Q K^T
+    static constexpr int kStepsPV = 128 * EB / 32;               // product instructions of O += P V (128 keys)
+    static constexpr int kVStepBytes = (32 / EB) * 128;          // V rows (keys) of one instruction x 128 bytes
+    static constexpr int kPCols = 128 * EB / 4;                  // tensor-memory columns of P (packed)
     static constexpr int kPanelBytes = 128 * 128;                // 128 rows x 128 bytes
     static constexpr int kTileBytes = kPanels * kPanelBytes;     // one Q / K / V tile
     static constexpr int kStages = (D == 128) ? 4 : 6;           // K/V ring
@@ -119,21 +128,59 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_
         : "memory");
 }
 // Same with ready-made 64-bit descriptors: one instruction per product, nothing to compute at issue time
+template <int EB = 2>
 __device__ __forceinline__ void mma_ss64(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                          uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
+    if constexpr (EB == 2) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
 }
+template <int EB = 2>
 __device__ __forceinline__ void mma_ts64(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
                                          uint32_t accumulate) {
+    if constexpr (EB == 2) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], [%1], %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
+}
+// 16 consecutive 32-bit columns of this thread's tensor-memory lane
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(taddr)
         : "memory");
+}
+// four fp32 -> four E4M3 codes (round to nearest even, saturating at +-448), first argument in the low byte
+__device__ __forceinline__ uint32_t pack_e4m3x4(float a, float b, float c, float d) {
+    uint32_t r;
+    asm("{\n\t.reg .b16 lo, hi;\n\t"
+        "cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1;\n\t"
+        "cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3;\n\t"
+        "mov.b32 %0, {lo, hi};\n\t}"
+        : "=r"(r) : "f"(a), "f"(b), "f"(c), "f"(d));
+    return r;
 }
 __device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | lo; }
 // 32 consecutive 32-bit columns of this thread's tensor-memory lane
@@ -177,10 +224,13 @@ __device__ __forceinline__ uint32_t smem_desc_lo(uint32_t saddr, uint32_t lbo) {
 __host__ __device__ constexpr uint32_t smem_desc_hi(uint32_t sbo) {
     return (sbo >> 4) | (1u << 14) | (2u << 29);
 }
-// Instruction descriptor: bf16 x bf16 -> fp32, A K-major, B K-major (b_mn = 0) or MN-major (1).
-__host__ __device__ constexpr uint32_t make_idesc(int M, int N, int b_mn) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(N >> 3) << 17) |
-           ((uint32_t)(M >> 4) << 24);
+// Instruction descriptor: bf16 x bf16 -> fp32 (operand format code 1 of kind::f16) or
+// E4M3 x E4M3 -> fp32 (format code 0 of kind::f8f6f4); A K-major, B K-major (b_mn = 0) or
+// MN-major (1).  Bits: 4-5 accumulator format (1 = fp32), 7-9 A format, 10-12 B format,
+// 16 B major, 17-22 N / 8, 24-28 M / 16.
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N, int b_mn, int eb = 2) {
+    return (1u << 4) | ((eb == 2 ? 1u : 0u) << 7) | ((eb == 2 ? 1u : 0u) << 10) | ((uint32_t)b_mn << 16) |
+           ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
 struct PrefillParams {
@@ -230,11 +280,11 @@ __device__ __forceinline__ uint32_t elect_one() {
     return pred;
 }
 
-template <int D>
+template <int D, int EB = 2>
 __global__ void __launch_bounds__(512, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, const PrefillParams prm) {
-    using C = PrefillCfg<D>;
+    using C = PrefillCfg<D, EB>;
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment for the swizzled tiles
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -329,7 +379,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     ++n_q[i];
                     mbar_arrive_expect_tx(&q_full[i], C::kTileBytes);
                     for (int p = 0; p < C::kPanels; ++p)
-                        tma_load_3d(sQ + i * C::kTileBytes + p * C::kPanelBytes, &map_q, p * 64, q0 + i * 128, bh,
+                        tma_load_3d(sQ + i * C::kTileBytes + p * C::kPanelBytes, &map_q, p * C::kPanelCols, q0 + i * 128, bh,
                                     &q_full[i]);
                 }
                 for (int t = 0; t < T; ++t) {
@@ -340,7 +390,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         mbar_arrive_expect_tx(&kv_full[stage], C::kTileBytes);
                         for (int p = 0; p < C::kPanels; ++p)
                             tma_load_3d(sKV + stage * C::kTileBytes + p * C::kPanelBytes, kv == 0 ? &map_k : &map_v,
-                                        p * 64, t * 128, bh, &kv_full[stage]);
+                                        p * C::kPanelCols, t * 128, bh, &kv_full[stage]);
                     }
                 }
             }
@@ -354,8 +404,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         reg_dec<96>();
         {
             const uint32_t leader = elect_one();
-            constexpr uint32_t idesc_s = make_idesc(128, 128, 0);
-            constexpr uint32_t idesc_o = make_idesc(128, D, 1);
+            constexpr uint32_t idesc_s = make_idesc(128, 128, 0, EB);
+            constexpr uint32_t idesc_o = make_idesc(128, D, 1, EB);
             const uint32_t tS[2] = {tmem_base + C::kColS0, tmem_base + C::kColS1};
             const uint32_t tO[2] = {tmem_base + C::kColO0, tmem_base + C::kColO1};
             const uint32_t tP[2] = {tmem_base + C::kColP0, tmem_base + C::kColP1};
@@ -366,7 +416,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             const uint32_t q_lo[2] = {smem_desc_lo(smem_u32(sQ), 16), smem_desc_lo(smem_u32(sQ + C::kTileBytes), 16)};
             const uint32_t k_lo0 = smem_desc_lo(smem_u32(sKV), 16);
             const uint32_t v_lo0 = smem_desc_lo(smem_u32(sKV), C::kPanelBytes);
-            constexpr int KS = D / 16;
+            constexpr int KS = C::kStepsS;
+            constexpr int KP = C::kStepsPV;
             constexpr int LA = C::kLookahead;
             auto koff = [](int ks) -> uint32_t { return (uint32_t)(((ks >> 2) * C::kPanelBytes + (ks & 3) * 32) >> 4); };
             // products of one batch; mid(ks) runs on all lanes after product ks
@@ -374,26 +425,27 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 const uint32_t ka = k_lo0 + stage * (C::kTileBytes >> 4);
 #pragma unroll
                 for (int ks = 0; ks < KS; ++ks) {
-                    if (leader) mma_ss64(tS[i], desc64(q_lo[i] + koff(ks), desc_hi), desc64(ka + koff(ks), desc_hi), idesc_s, ks > 0);
+                    if (leader) mma_ss64<EB>(tS[i], desc64(q_lo[i] + koff(ks), desc_hi), desc64(ka + koff(ks), desc_hi), idesc_s, ks > 0);
                     __syncwarp();
                     mid(ks * (8 / KS));
                 }
             };
-            auto fire_PV_part = [&](int i, int stage, bool first, int ks0) {
+            auto fire_PV_part = [&](int i, int stage, bool first, int part) {      // keys 64*part .. 64*part+63
                 const uint32_t va = v_lo0 + stage * (C::kTileBytes >> 4);
 #pragma unroll
-                for (int ks = ks0; ks < ks0 + 4; ++ks) {
-                    if (leader) mma_ts64(tO[i], tP[i] + ks * 8, desc64(va + ks * (2048 >> 4), desc_hi), idesc_o, (!first) || ks > 0);
+                for (int kk = 0; kk < KP / 2; ++kk) {
+                    const int ks = part * (KP / 2) + kk;
+                    if (leader) mma_ts64<EB>(tO[i], tP[i] + ks * 8, desc64(va + ks * (C::kVStepBytes >> 4), desc_hi), idesc_o, (!first) || ks > 0);
                     __syncwarp();
                 }
             };
             auto fire_PV = [&](int i, int stage, bool first, auto&& mid) {
                 const uint32_t va = v_lo0 + stage * (C::kTileBytes >> 4);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    if (leader) mma_ts64(tO[i], tP[i] + ks * 8, desc64(va + ks * (2048 >> 4), desc_hi), idesc_o, (!first) || ks > 0);
+                for (int ks = 0; ks < KP; ++ks) {
+                    if (leader) mma_ts64<EB>(tO[i], tP[i] + ks * 8, desc64(va + ks * (C::kVStepBytes >> 4), desc_hi), idesc_o, (!first) || ks > 0);
                     __syncwarp();
-                    mid(ks);
+                    mid(ks * (8 / KP));
                 }
             };
             auto commit = [&](uint64_t* bar) {
@@ -453,7 +505,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         if (!pf_wait(&p_full[0], n_p0 & 1, kWaitPFull, abort_flag)) goto done;
                         e_pf0 = 0; ++n_p0;
                         tc_fence_after();
-                        fire_PV_part(0, st_v, false, 4);
+                        fire_PV_part(0, st_v, false, 1);
                         commit(&pv_done[0]);
                     } else if (pv0) {
                         if (!e_pf0 && !pf_wait(&p_full[0], n_p0 & 1, kWaitPFull, abort_flag)) goto done;
@@ -493,7 +545,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         if (!pf_wait(&p_full[1], n_p1 & 1, kWaitPFull, abort_flag)) goto done;
                         e_pf1 = 0; ++n_p1;
                         tc_fence_after();
-                        fire_PV_part(1, st_v, false, 4);
+                        fire_PV_part(1, st_v, false, 1);
                         commit(&pv_done[1]);
                     } else if (pv1) {
                         if (!e_pf1 && !pf_wait(&p_full[1], n_p1 & 1, kWaitPFull, abort_flag)) goto done;
@@ -550,6 +602,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             const int limit = prm.causal ? min(Nk, gi + 1) : Nk;   // keys [0, limit) are visible
             float L = -INFINITY;                       // log2-domain state: L = (s_i - ln w_i) * log2(e)
             float inv_l = 1.f;                         // 1 / l of the previous tile
+            float K_prev = 0.f;                        // exponent offset of the stored weights (E4M3 only)
             for (int t = 0; t < Ti; ++t) {
                 if (!pf_wait(&s_full[i], n_s & 1, kWaitSFull, abort_flag)) goto done;
                 ++n_s;
@@ -595,17 +648,31 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 // the order of the products (S(t) is issued after P V(t-1), which needed the
                 // correction of step t-1).  With lookahead 2 S(t) runs ahead, so the message is
                 // posted below, after the wait for P V(t-1) that the P store needs anyway.
-                const float beta = e_old * inv_l;
+                float beta = e_old * inv_l;
+                // E4M3 weights: in this form the weights of a late tile are small against the mass
+                // already accumulated (x_j = s_j - L_{t-1} is far below zero on long rows), below
+                // E4M3's normal range (2^-6).  They are therefore stored times 2^K, K chosen per row
+                // and tile so that the tile's largest weight lands in [2^7, 2^8): an exact power of
+                // two that rides in the exponent of the exponential, is taken out of the row sum
+                // again, and reaches the accumulator through the factor beta (2^(K_t - K_{t-1})) and
+                // the final reciprocal (2^-K_T).  K is capped at 64: a tile whose largest weight is
+                // below 2^-57 of the accumulated mass is lost in fp32 anyway.
+                float Kf = 0.f;
+                if constexpr (EB == 1) {
+                    Kf = fminf(floorf(ref - m0 * c) + 7.f, 64.f);
+                    beta *= ex2(Kf - K_prev);
+                    K_prev = Kf;
+                }
                 if (C::kLookahead == 1 && t > 0) {
                     sAlpha[(n_ae & 1) * 256 + i * 128 + row] = beta;
                     ++n_ae;
                     mbar_arrive(&alpha_full[i]);
                 }
-                const uint64_t c2 = pack2(c, c), nref2 = pack2(-ref, -ref);
+                const uint64_t c2 = pack2(c, c), nref2 = pack2(Kf - ref, Kf - ref);
                 uint64_t acc0 = pack2(0.f, 0.f), acc1 = acc0;
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    uint32_t pk[32];
+                    uint32_t pk[C::kPCols / 2];     // the weights of 64 keys, packed
 #pragma unroll
                     for (int j = 0; j < 64; j += 4) {
                         if (C::kLookahead == 1 && h == 1 && j == 32) {
@@ -620,8 +687,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
                         acc0 = add2(acc0, pack2(p0, p1));
                         acc1 = add2(acc1, pack2(p2, p3));
-                        pk[j / 2] = pack_bf16x2(p0, p1);
-                        pk[j / 2 + 1] = pack_bf16x2(p2, p3);
+                        if constexpr (EB == 2) {
+                            pk[j / 2] = pack_bf16x2(p0, p1);
+                            pk[j / 2 + 1] = pack_bf16x2(p2, p3);
+                        } else {
+                            pk[j / 4] = pack_e4m3x4(p0, p1, p2, p3);
+                        }
                     }
                     if (C::kLookahead > 1 && h == 0 && n_pk > 0) {
                         // P has a region of its own: the previous P V must have read it
@@ -633,13 +704,16 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                             mbar_arrive(&alpha_full[i]);
                         }
                     }
-                    tmem_st32(tP + 32 * h, pk);
+                    if constexpr (EB == 2) tmem_st32(tP + 32 * h, pk);
+                    else tmem_st16(tP + 16 * h, pk);
                 }
                 ++n_pk;
                 float a0, a1, a2, a3;
                 unpack2(acc0, a0, a1);
                 unpack2(acc1, a2, a3);
-                const float l = e_old + ((a0 + a1) + (a2 + a3));
+                float rowsum = (a0 + a1) + (a2 + a3);
+                if constexpr (EB == 1) rowsum *= ex2(-Kf);
+                const float l = e_old + rowsum;
                 inv_l = rcp(l);                              // the hidden division: one reciprocal per row and tile
                 L = ref + lg2(l);
                 tc_wait_st();
@@ -652,7 +726,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 // that follows from the product order; a one-tile item waits for its own P V,
                 // which is issued only after the previous epilogue has released O.
                 if (Ti == 1 && !pf_wait(&pv_done[i], (n_pk - 1) & 1, kWaitPVDone, abort_flag)) goto done;
-                sFinal[i * 128 + row] = inv_l;
+                sFinal[i * 128 + row] = (EB == 1) ? inv_l * ex2(-K_prev) : inv_l;
                 mbar_arrive(&final_full[i]);
             }
             if (prm.lse != nullptr && Ti > 0 && gi < Nq) prm.lse[(long long)bh * Nq + gi] = L * kLn2;
