@@ -272,7 +272,7 @@ def make_sets(w, device, min_bytes):
     return sets, set_bytes
 
 
-def bench_workload(fd, w, steps, warmup, torch, device):
+def bench_workload(fd, w, steps, warmup, torch, device, e4m3=False):
     """Device-resident timing of one workload; returns a dict of results."""
     sc = f32(w.scale)
     if w.splitk:
@@ -289,7 +289,14 @@ def bench_workload(fd, w, steps, warmup, torch, device):
                 "gbs": alg_bytes * steps / (ms * 1e-3) / 1e9, "launches": launches, "num_splits": S,
                 "l2": "inputs (34 GB) exceed L2", "tensors": (q, k, v, o)}
     sets, set_bytes = make_sets(w, device, 1.5 * L2_BYTES)
-    fn = lambda i: fd.flashd_attn_fwd(*sets[i % len(sets)][:3], sc, w.causal, o=sets[i % len(sets)][3])
+    if e4m3:
+        # the same tensors stored as FP8-E4M3 (the paper's second format), bf16 output
+        sets = [(q.to(torch.float8_e4m3fn), k.to(torch.float8_e4m3fn), v.to(torch.float8_e4m3fn), o)
+                for (q, k, v, o) in sets]
+        set_bytes = set_bytes * 5 // 8
+        fn = lambda i: fd.flashd_attn_fwd_fp8(*sets[i % len(sets)][:3], sc, w.causal, o=sets[i % len(sets)][3])
+    else:
+        fn = lambda i: fd.flashd_attn_fwd(*sets[i % len(sets)][:3], sc, w.causal, o=sets[i % len(sets)][3])
     n0 = fd.launch_count()
     ms = time_gpu(fn, steps, warmup, torch)
     launches = (fd.launch_count() - n0) * steps // (steps + warmup)
@@ -685,6 +692,22 @@ def main():
                     r["frac_tensor_measured"] = r["tflops"] / peaks["bf16_tflops"]
                     r["frac_tensor_nominal"] = r["tflops"] / NOMINAL_BF16_TFLOPS
                 others[name] = r
+                torch.cuda.empty_cache()
+            # configurations 2 and 3 with E4M3 operands on the tensor path; the peak of that
+            # dtype is the measured bf16 figure times the nominal ratio of 2
+            for name in ("c2", "c3"):
+                ow = synth.WORKLOADS[name]
+                smp = ClockSampler(local_rank)
+                smp.start()
+                smp.mark_start()
+                r = bench_workload(fd, ow, 30 if name == "c3" else 200, 3, torch, device, e4m3=True)
+                smp.mark_end()
+                r["clocks"] = smp.stop()
+                r.pop("tensors", None)
+                r["dtype"] = "e4m3 operands, fp32 accumulate, bf16 output"
+                r["frac_tensor_measured"] = r["tflops"] / (2 * peaks["bf16_tflops"])
+                r["frac_tensor_nominal"] = r["tflops"] / (2 * NOMINAL_BF16_TFLOPS)
+                others[name + "_e4m3"] = r
                 torch.cuda.empty_cache()
         except Exception as ex:  # the headline number stands on its own
             others["error"] = repr(ex)
