@@ -34,7 +34,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (c4: a batch-4 capture scaled by 16, traffic being
 # proportional to the bytes streamed).  Must be set back to None when that kernel changes.
-NCU_TRAFFIC_BYTES = {"c1": 38.1e6, "c2": 589.2e6, "c3": None, "c4": 34.51e9}
+NCU_TRAFFIC_BYTES = {"c1": 38.1e6, "c2": 589.2e6, "c3": None, "c4": 34.51e9, "c2_e4m3": 194.8e6}
 
 
 def f32(x: float) -> float:
@@ -514,6 +514,9 @@ def main():
                     help="print the output error of the PWL / confined-range datapath model (Sec. IV-B) instead of timing")
     ap.add_argument("--gqa", action="store_true",
                     help="time the decode variants (config 4 with shared K/V heads; config 4 with FP8-E4M3 K/V) instead")
+    ap.add_argument("--e4m3", action="store_true",
+                    help="time the workload (c2 or c3, d = 128) with FP8-E4M3 operands on the tensor path; no "
+                         "end-to-end leg (the host entry point takes bf16 / fp32)")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the workload's batch size B (smaller case for profiler captures)")
     args = ap.parse_args()
@@ -568,6 +571,14 @@ def main():
     else:
         sets, set_bytes = make_sets(w, device, 1.5 * L2_BYTES)
         step = lambda i: fd.flashd_attn_fwd(*sets[i % len(sets)][:3], sc, w.causal, o=sets[i % len(sets)][3])
+        if args.e4m3:
+            if w.d != 128:
+                raise SystemExit("--e4m3 needs a workload with d = 128 (c2, c3)")
+            sets = [(q.to(torch.float8_e4m3fn), k.to(torch.float8_e4m3fn), v.to(torch.float8_e4m3fn), o)
+                    for (q, k, v, o) in sets]
+            set_bytes = set_bytes * 5 // 8
+            step = lambda i: fd.flashd_attn_fwd_fp8(*sets[i % len(sets)][:3], sc, w.causal, o=sets[i % len(sets)][3])
+            args.no_e2e = True
         l2_note = f"rotating {len(sets)} input sets of {set_bytes / 1e6:.0f} MB each (> 126 MB L2 in total)"
     sampler.start()
     for i in range(args.warmup):
@@ -608,18 +619,26 @@ def main():
                 "kernel": "splitk_partial_kernel (+combine, timed together)"}
     else:
         achieved = w.flops / (local_ms / args.steps * 1e-3) / 1e12
-        roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["bf16_tflops"], "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if args.batch == 0 else None,
-                "peak_source": peaks["source"],
-                "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS, "kernel": f"prefill_kernel<{w.d}>"}
+        # E4M3 products: the peak of that dtype = the measured bf16 figure x the nominal ratio of 2
+        pk_scale = 2.0 if args.e4m3 else 1.0
+        traffic = NCU_TRAFFIC_BYTES.get(args.workload + ("_e4m3" if args.e4m3 else "")) if args.batch == 0 else None
+        roof = {"bound": "tensor", "achieved": achieved, "peak": pk_scale * peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": achieved / (pk_scale * peaks["bf16_tflops"]), "traffic": traffic,
+                "peak_source": peaks["source"] + (" bf16 x 2 (nominal fp8 : bf16 ratio)" if args.e4m3 else ""),
+                "frac_of_nominal": achieved / (pk_scale * NOMINAL_BF16_TFLOPS),
+                "kernel": f"prefill_kernel<{w.d}, 1>" if args.e4m3 else f"prefill_kernel<{w.d}>"}
 
     line = {
         "metric": "attn_fwd_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "vs_baseline": None, "dtype": "e4m3" if args.e4m3 else "bf16", "data": "synthetic",
         "config": workload_config(w, {"l2": l2_note, "parallelism": "replicas only" if world > 1 else "1 gpu"}),
         "roofline": roof, "clocks": clocks, "gpu_launches": int(launches),
     }
+
+    if args.e4m3:
+        line["config"]["in_dtype"] = "e4m3"
+        line["config"]["workload"] = line["config"]["workload"].replace(" bf16", "") + " (FP8-E4M3 operands)"
 
     if rank == 0 and world == 1 and not w.splitk:
         # launch gaps: the same launches replayed from a CUDA graph (50 per replay)

@@ -238,6 +238,20 @@ int flashd_attn_fwd_splitk_paged(const void* q, const void* k_pages, const void*
                                  void* workspace, size_t workspace_bytes,
                                  int B, int H, int Nq, int max_pages, int page_size, int num_pages,
                                  int d, float scale, int num_splits, void* stream);
+/* The same over a pool of FP8-E4M3 pages (one byte per element, widened exactly
+ * as in flashd_splitk_partial_fp8kv; q and o stay bf16).  A ring stage then
+ * holds twice the keys: page_size must be a multiple of 128 keys at d = 128
+ * and of 256 at d = 64.                                                     */
+int flashd_splitk_partial_paged_fp8kv(const void* q, const void* k_pages, const void* v_pages,
+                                      const int* block_table, const int* seq_lens,
+                                      void* workspace, size_t workspace_bytes,
+                                      int B, int H, int Nq, int max_pages, int page_size, int num_pages,
+                                      int d, float scale, int num_splits, void* stream);
+int flashd_attn_fwd_splitk_paged_fp8kv(const void* q, const void* k_pages, const void* v_pages, void* o,
+                                       const int* block_table, const int* seq_lens,
+                                       void* workspace, size_t workspace_bytes,
+                                       int B, int H, int Nq, int max_pages, int page_size, int num_pages,
+                                       int d, float scale, int num_splits, void* stream);
 
 /* ------------------------------------------------------------------------
  * Split-K forward with K and V stored as FP8-E4M3 (the second number format of

@@ -21,6 +21,7 @@ EXPORTED_SYMBOLS = (
     "flashd_gqa_num_splits", "flashd_gqa_partial", "flashd_attn_fwd_gqa", "flashd_attn_fwd_pwl",
     "flashd_splitk_partial_fp8kv", "flashd_attn_fwd_splitk_fp8kv",
     "flashd_splitk_partial_paged", "flashd_attn_fwd_splitk_paged", "flashd_attn_fwd_fp8",
+    "flashd_splitk_partial_paged_fp8kv", "flashd_attn_fwd_splitk_paged_fp8kv",
     "flashd_attn_fwd_host", "flashd_skip_stats", "flashd_last_device_status", "flashd_status_string", "flashd_version", "flashd_launch_count",
 )
 
@@ -65,6 +66,8 @@ def lib() -> ctypes.CDLL:
             L.flashd_attn_fwd_splitk.argtypes = [vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_splitk_partial_paged.argtypes = [vp, vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_attn_fwd_splitk_paged.argtypes = [vp, vp, vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, ci, ci, cf, ci, vp]
+            L.flashd_splitk_partial_paged_fp8kv.argtypes = L.flashd_splitk_partial_paged.argtypes
+            L.flashd_attn_fwd_splitk_paged_fp8kv.argtypes = L.flashd_attn_fwd_splitk_paged.argtypes
             fp = ctypes.POINTER(ctypes.c_float)
             L.flashd_attn_fwd_pwl.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, ci,
                                               ci, fp, fp, ci, fp, fp, cf, cf, ci, vp]
@@ -312,7 +315,8 @@ def flashd_splitk_partial_paged(q, k_pages, v_pages, block_table, seq_lens, scal
     B, H, Nq, d, num_pages, page_size, max_pages = _paged_dims(q, k_pages, v_pages, block_table, seq_lens)
     if workspace is None:
         workspace = torch.empty((B, H, Nq, num_splits, d + 1), dtype=torch.float32, device=q.device)
-    _check(lib().flashd_splitk_partial_paged(_ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(block_table), _ptr(seq_lens),
+    fn = lib().flashd_splitk_partial_paged_fp8kv if k_pages.dtype == torch.float8_e4m3fn else lib().flashd_splitk_partial_paged
+    _check(fn(_ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(block_table), _ptr(seq_lens),
                                              _ptr(workspace), workspace.numel() * workspace.element_size(), B, H, Nq,
                                              max_pages, page_size, num_pages, d, float(scale), int(num_splits),
                                              _stream_ptr(stream)), "flashd_splitk_partial_paged")
@@ -329,11 +333,10 @@ def flashd_attn_fwd_splitk_paged(q, k_pages, v_pages, block_table, seq_lens, sca
         workspace = torch.empty((B, H, Nq, max(S, 1), d + 1), dtype=torch.float32, device=q.device)
     if o is None:
         o = torch.empty_like(q)
-    _check(lib().flashd_attn_fwd_splitk_paged(_ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(o), _ptr(block_table),
-                                              _ptr(seq_lens), _ptr(workspace),
-                                              workspace.numel() * workspace.element_size(), B, H, Nq, max_pages,
-                                              page_size, num_pages, d, float(scale), int(num_splits),
-                                              _stream_ptr(stream)), "flashd_attn_fwd_splitk_paged")
+    fn = lib().flashd_attn_fwd_splitk_paged_fp8kv if k_pages.dtype == torch.float8_e4m3fn else lib().flashd_attn_fwd_splitk_paged
+    _check(fn(_ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(o), _ptr(block_table), _ptr(seq_lens), _ptr(workspace),
+              workspace.numel() * workspace.element_size(), B, H, Nq, max_pages, page_size, num_pages, d,
+              float(scale), int(num_splits), _stream_ptr(stream)), "flashd_attn_fwd_splitk_paged")
     return o
 
 

@@ -468,7 +468,7 @@ int flashd_attn_fwd_splitk_fp8kv(const void* q, const void* k, const void* v, vo
     return flashd_splitk_combine(workspace, o, nullptr, B, H, Nq, d, num_splits, FLASHD_BF16, stream);
 }
 
-int flashd_splitk_partial_paged(const void* q, const void* k_pages, const void* v_pages, const int* block_table,
+static int splitk_partial_paged_impl(int kvb, const void* q, const void* k_pages, const void* v_pages, const int* block_table,
                                 const int* seq_lens, void* workspace, size_t workspace_bytes, int B, int H, int Nq,
                                 int max_pages, int page_size, int num_pages, int d, float scale, int num_splits,
                                 void* stream) {
@@ -481,7 +481,7 @@ int flashd_splitk_partial_paged(const void* q, const void* k_pages, const void* 
         (reinterpret_cast<uintptr_t>(block_table) & 3u) || (reinterpret_cast<uintptr_t>(seq_lens) & 3u))
         return FLASHD_ERR_ALIGN;
     if (d != 128 && d != 64) return FLASHD_ERR_UNSUPPORTED;
-    const int chunk = (d == 128) ? DecodeCfg<128>::kChunk : DecodeCfg<64>::kChunk;
+    const int chunk = 16384 / (d * kvb);                           // keys per ring stage (DecodeCfg::kChunk)
     if (page_size % chunk != 0) return FLASHD_ERR_UNSUPPORTED;     // a ring stage must not straddle pages
     if (num_splits < 1 || num_splits > FLASHD_MAX_SPLITS) return FLASHD_ERR_WORKSPACE;
     if (workspace_bytes < flashd_splitk_workspace_bytes(B, H, Nq, d, num_splits)) return FLASHD_ERR_WORKSPACE;
@@ -494,9 +494,29 @@ int flashd_splitk_partial_paged(const void* q, const void* k_pages, const void* 
     pg.page_size = page_size;
     pg.num_pages = num_pages;
     pg.H = H;
-    if (d == 128)
-        return launch_partial<128, 2, true>(q, k_pages, v_pages, workspace, rows, Nq, 0, scale, num_splits, as_stream(stream), pg);
-    return launch_partial<64, 2, true>(q, k_pages, v_pages, workspace, rows, Nq, 0, scale, num_splits, as_stream(stream), pg);
+    cudaStream_t s = as_stream(stream);
+    if (kvb == 2) {
+        if (d == 128) return launch_partial<128, 2, true>(q, k_pages, v_pages, workspace, rows, Nq, 0, scale, num_splits, s, pg);
+        return launch_partial<64, 2, true>(q, k_pages, v_pages, workspace, rows, Nq, 0, scale, num_splits, s, pg);
+    }
+    if (d == 128) return launch_partial<128, 1, true>(q, k_pages, v_pages, workspace, rows, Nq, 0, scale, num_splits, s, pg);
+    return launch_partial<64, 1, true>(q, k_pages, v_pages, workspace, rows, Nq, 0, scale, num_splits, s, pg);
+}
+
+int flashd_splitk_partial_paged(const void* q, const void* k_pages, const void* v_pages, const int* block_table,
+                                const int* seq_lens, void* workspace, size_t workspace_bytes, int B, int H, int Nq,
+                                int max_pages, int page_size, int num_pages, int d, float scale, int num_splits,
+                                void* stream) {
+    return splitk_partial_paged_impl(2, q, k_pages, v_pages, block_table, seq_lens, workspace, workspace_bytes, B, H, Nq,
+                                     max_pages, page_size, num_pages, d, scale, num_splits, stream);
+}
+
+int flashd_splitk_partial_paged_fp8kv(const void* q, const void* k_pages, const void* v_pages, const int* block_table,
+                                      const int* seq_lens, void* workspace, size_t workspace_bytes, int B, int H,
+                                      int Nq, int max_pages, int page_size, int num_pages, int d, float scale,
+                                      int num_splits, void* stream) {
+    return splitk_partial_paged_impl(1, q, k_pages, v_pages, block_table, seq_lens, workspace, workspace_bytes, B, H, Nq,
+                                     max_pages, page_size, num_pages, d, scale, num_splits, stream);
 }
 
 int flashd_attn_fwd_splitk_paged(const void* q, const void* k_pages, const void* v_pages, void* o,
@@ -509,6 +529,21 @@ int flashd_attn_fwd_splitk_paged(const void* q, const void* k_pages, const void*
         (long long)max_pages * page_size <= 0x7fffffffLL)
         num_splits = flashd_splitk_num_splits(B, H, Nq, max_pages * page_size, d);
     const int st = flashd_splitk_partial_paged(q, k_pages, v_pages, block_table, seq_lens, workspace, workspace_bytes,
+                                               B, H, Nq, max_pages, page_size, num_pages, d, scale, num_splits, stream);
+    if (st != FLASHD_OK) return st;
+    return flashd_splitk_combine(workspace, o, nullptr, B, H, Nq, d, num_splits, FLASHD_BF16, stream);
+}
+
+int flashd_attn_fwd_splitk_paged_fp8kv(const void* q, const void* k_pages, const void* v_pages, void* o,
+                                 const int* block_table, const int* seq_lens, void* workspace,
+                                 size_t workspace_bytes, int B, int H, int Nq, int max_pages, int page_size,
+                                 int num_pages, int d, float scale, int num_splits, void* stream) {
+    if (!o) return FLASHD_ERR_NULL;
+    if (!aligned16(o)) return FLASHD_ERR_ALIGN;
+    if (num_splits <= 0 && B > 0 && H > 0 && Nq > 0 && max_pages > 0 && page_size > 0 &&
+        (long long)max_pages * page_size <= 0x7fffffffLL)
+        num_splits = flashd_splitk_num_splits(B, H, Nq, max_pages * page_size, d);
+    const int st = flashd_splitk_partial_paged_fp8kv(q, k_pages, v_pages, block_table, seq_lens, workspace, workspace_bytes,
                                                B, H, Nq, max_pages, page_size, num_pages, d, scale, num_splits, stream);
     if (st != FLASHD_OK) return st;
     return flashd_splitk_combine(workspace, o, nullptr, B, H, Nq, d, num_splits, FLASHD_BF16, stream);

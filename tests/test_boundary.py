@@ -83,6 +83,13 @@ def test_validation_happens_before_any_launch(flashd_lib):
     assert pp(a, a, a, a, a, a, ws_need - 1, 1, 1, 1, 4, 64, 8, 128, 0.1, 4, None) == 5
     assert pp(a, a, a, a, a, a, ws_need, 1, 1, 1, 4, 64, 8, 128, 0.1, 65, None) == 5
     assert L.flashd_attn_fwd_splitk_paged(a, a, a, null, a, a, a, ws_need, 1, 1, 1, 4, 64, 8, 128, 0.1, 4, None) == 1
+    assert L.flashd_splitk_partial_paged_fp8kv(a, a, a, a, a, a, ws_need, 1, 1, 1, 4, 64, 8, 128, 0.1, 4, None) == 3   # E4M3 stage = 128 keys
+    # E4M3 operands on the tensor path: (q, k, v, o, lse, out_dtype, B, H, Nq, Nk, d, scale, causal)
+    o2 = ctypes.c_void_p(a.value + 512)
+    assert L.flashd_attn_fwd_fp8(a, a, a, o2, None, 0, 1, 1, 8, 8, 64, 0.1, 0, None) == 3
+    assert L.flashd_attn_fwd_fp8(a, a, a, o2, None, 7, 1, 1, 8, 8, 128, 0.1, 0, None) == 3
+    assert L.flashd_attn_fwd_fp8(a, a, a, a, None, 0, 1, 1, 8, 8, 128, 0.1, 0, None) == 2     # o aliases q
+    assert L.flashd_attn_fwd_fp8(null, a, a, o2, None, 0, 1, 1, 8, 8, 128, 0.1, 0, None) == 1
     assert L.flashd_attn_fwd_host(a, a, a, a, 7, 1, 1, 8, 8, 64, 0.1, 0, None) == 3
     assert L.flashd_attn_fwd_host(a, a, a, a, 2, 1, 1, 8, 8, 64, 0.1, 1, None) == 3  # split-K is non-causal
     assert flashd_lib.launch_count() == n0

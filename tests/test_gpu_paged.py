@@ -116,3 +116,31 @@ def test_bad_table_is_reported_not_followed(flashd_lib):
     st, detail = flashd_lib.flashd_last_device_status()
     assert st == 0, detail
     check(got, q, ks, vs, [200, 100], sc, "after bad tables")
+
+
+@pytest.mark.parametrize("d,page_size,lens,H,Nq,splits", [
+    (128, 128, [1, 127, 128, 129, 3000], 3, 1, 0),
+    (128, 256, [5000, 0, 600], 2, 2, 3),
+    (64, 256, [255, 256, 257, 2000], 3, 1, 0),
+])
+def test_paged_fp8_pool_matches_oracle(flashd_lib, d, page_size, lens, H, Nq, splits):
+    """The pool stored as FP8-E4M3: the oracle takes the stored values widened exactly."""
+    F8 = torch.float8_e4m3fn
+    sc = f32_scale(d)
+    k_pages, v_pages, table, seq_lens, ks, vs = build_pool(lens, H, d, page_size, seed=3 + d + page_size)
+    k_pages = (k_pages.float() / 30).to(F8)       # the garbage of unowned pages stays large against the keys
+    v_pages = (v_pages.float() / 30).to(F8)
+    ks = [x.to(F8) for x in ks]
+    vs = [x.to(F8) for x in vs]
+    # owned keys must be the E4M3 rounding of the sequences' keys, whatever the pool held before
+    for b, n in enumerate(lens):
+        for p in range((n + page_size - 1) // page_size):
+            m = min(page_size, n - p * page_size)
+            k_pages[table[b, p], :, :m] = ks[b][:, p * page_size:p * page_size + m]
+            v_pages[table[b, p], :, :m] = vs[b][:, p * page_size:p * page_size + m]
+    q, _, _ = synth.random_qkv(len(lens), H, Nq, 1, d, seed=98)
+    got = flashd_lib.flashd_attn_fwd_splitk_paged(q.cuda(), k_pages.cuda(), v_pages.cuda(), table.cuda(),
+                                                  seq_lens.cuda(), sc, splits)
+    st, detail = flashd_lib.flashd_last_device_status()
+    assert st == 0, detail
+    check(got, q, ks, vs, lens, sc, ("fp8", d, page_size))
