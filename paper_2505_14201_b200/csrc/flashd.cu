@@ -117,7 +117,24 @@ int launch_prefill(const void* q, const void* k, const void* v, void* o, float* 
     const int sms = sm_count();
     if (sms <= 0) return FLASHD_ERR_CUDA;
     const int grid = prm.n_work < sms ? prm.n_work : sms;
-    prefill_kernel<D, EB><<<grid, C::kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, prm);
+    // launched with programmatic stream serialisation: the grid may be set up while the previous
+    // kernel of the stream drains (the kernel itself waits for that kernel before it reads or writes
+    // global memory)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)C::kThreads);
+    cfg.dynamicSmemBytes = C::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, prefill_kernel<D, EB>, mq, mk, mv, prm) != cudaSuccess) {
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        cudaGetLastError();
+        return FLASHD_ERR_CUDA;
+    }
     return after_launch();
 }
 

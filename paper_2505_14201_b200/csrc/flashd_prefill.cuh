@@ -343,6 +343,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // Programmatic dependent launch: the set-up above may run while the previous kernel of the
+    // stream drains; nothing of global memory is touched before that kernel has completed and its
+    // writes are visible.  The next kernel of the stream is released in the same way when every
+    // CTA of this grid has begun its last work item (it waits for this grid to complete before
+    // it touches memory).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const int Nq = prm.Nq, Nk = prm.Nk;
     const int n_kt_all = (Nk + 127) >> 7;
@@ -368,6 +374,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             uint32_t kv_it = 0;
             uint32_t n_q[2] = {0, 0};     // uses of each Q buffer so far
             for (int nw = 0, w = work_index(0); w < prm.n_work; w = work_index(++nw)) {
+                if (work_index(nw + 1) >= prm.n_work) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
                 const int qpair = prm.n_qpairs - 1 - w / prm.BH;
                 const int bh = w % prm.BH;
                 const int q0 = qpair * 256;
