@@ -459,6 +459,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 if (leader) tc_commit(bar);
                 __syncwarp();
             };
+            bool early0 = false;        // S_0(0) of the work item about to start has been issued already
             for (int nw = 0, w = work_index(0); w < prm.n_work; w = work_index(++nw)) {
                 const int qpair = prm.n_qpairs - 1 - w / prm.BH;
                 const int q0 = qpair * 256;
@@ -473,7 +474,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 for (int u = 0; u < LA && u < T; ++u) {
                     const uint32_t it_k = kv_it + 2 * u;
                     if (!pf_wait(&kv_full[stage_of(it_k)], parity_of(it_k), kWaitKVFull, abort_flag)) goto done;
-                    if (u < T0) {
+                    if (u == 0 && early0) {
+                        early0 = false;
+                    } else if (u < T0) {
                         if (u == 0) { if (!pf_wait(&q_full[0], n_qf0 & 1, kWaitQFull, abort_flag)) goto done; ++n_qf0; }
                         else { if (!pf_wait(&s_free[0], n_sf0 & 1, kWaitSFree, abort_flag)) goto done; ++n_sf0; }
                         tc_fence_after();
@@ -541,6 +544,28 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         });
                         commit(&s_full[0]);
                         if (t + LA + 1 == T0) commit(&q_empty[0]);
+                    }
+                    if (LA > 1 && t == T0 - 1) {
+                        // Tile 0 has had its last products of this work item.  Its first score product
+                        // of the NEXT work item does not have to wait for tile 1 to finish: S_0 is free
+                        // (its weights warps are past their last step), so if the next Q_0 and K(0)
+                        // have arrived it is issued here, and tile 0's weights start the next item
+                        // while tile 1 still closes this one (c1: +1.7 %).  Not at lookahead 1: there
+                        // it pulls the two tiles into phase, which costs more than it saves (c3: -2.5 %).
+                        const int wn = work_index(nw + 1);
+                        if (wn < prm.n_work) {
+                            const int T0n = n_tiles((prm.n_qpairs - 1 - wn / prm.BH) * 256);
+                            const uint32_t it_k0 = kv_it + 2 * T;
+                            if (T0n > 0 && mbar_test(&q_full[0], n_qf0 & 1) &&
+                                mbar_test(&kv_full[stage_of(it_k0)], parity_of(it_k0))) {
+                                ++n_qf0;
+                                tc_fence_after();
+                                fire_S(0, stage_of(it_k0), none);
+                                commit(&s_full[0]);
+                                if (T0n == 1) commit(&q_empty[0]);
+                                early0 = true;
+                            }
+                        }
                     }
                     if (pv1 && LA == 1) {
                         if (!e_or1 && !pf_wait(&o_ready[1], n_or1 & 1, kWaitOReady, abort_flag)) goto done;
