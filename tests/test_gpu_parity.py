@@ -388,3 +388,37 @@ def test_host_entry_point_pipelined_chunks(flashd_lib):
         want = oracle.attn_naive(q[b:b + 1, h:h + 1], k[b:b + 1, h:h + 1], v[b:b + 1, h:h + 1], sc, False)
         check_bf16(got[b:b + 1, h:h + 1], want, (b, h))
     ok_status(flashd_lib)
+
+
+def test_back_to_back_launches_see_each_others_output(flashd_lib):
+    """The tiled kernel is launched so that its set-up may overlap the drain of the previous kernel
+    of the stream.  A chain in which every forward takes the previous output as its V (no host
+    synchronisation in between) must equal the same chain run with a synchronisation after every
+    launch, and its last link must be right."""
+    for d, causal in ((64, False), (128, True)):
+        q, k, v = synth.random_qkv(2, 5, 512, 512, d, seed=61 + d)
+        sc = f32_scale(d)
+        qc, kc = q.cuda(), k.cuda()
+
+        def chain(sync):
+            x = v.cuda()
+            for _ in range(6):
+                x = flashd_lib.flashd_attn_fwd(qc, kc, x, sc, causal)
+                if sync:
+                    torch.cuda.synchronize()
+            torch.cuda.synchronize()
+            return x
+
+        a = chain(False)
+        b = chain(True)
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16)), (d, causal)
+        # last link against the oracle, from the fifth output
+        x = v.cuda()
+        for _ in range(5):
+            x = flashd_lib.flashd_attn_fwd(qc, kc, x, sc, causal)
+        want = oracle.attn_naive(q, k, x.cpu(), sc, causal)
+        err = np.abs(a.double().cpu().numpy() - want)
+        assert err.mean() <= BF16_MEAN, (d, causal, err.mean())
+        # a bf16 output above 2 in magnitude is on a grid coarser than the bound (see the module docstring)
+        assert err[np.abs(want) < 2.0].max() <= BF16_MAX, (d, causal)
+    ok_status(flashd_lib)
