@@ -33,6 +33,8 @@
 // Tensor memory (512 columns), D = 128: S0 | S1 | O0 | O1, P_i overlays the first 64
 // columns of S_i as packed bf16 pairs and is handed to the P V product in two halves of 64
 // keys; D = 64: S0 | S1 | P0 | P1 | O0 | O1.
+// Operands: bf16 (tcgen05.mma kind::f16) or FP8-E4M3 (kind::f8f6f4, D = 128; the weights are then
+// stored as E4M3 with a per-row power-of-two scale, see the weights warps).
 // Every mbarrier wait is bounded; a wait that runs out records itself in the
 // device status word, raises the CTA's abort flag and the CTA drains and exits.
 #pragma once
