@@ -308,6 +308,31 @@ int flashd_attn_fwd_gqa(const void* q, const void* k, const void* v, void* o,
                         int num_splits, void* stream);
 
 /* ------------------------------------------------------------------------
+ * Grouped-query decode over a paged K/V pool with one length per sequence:
+ * flashd_gqa_partial / flashd_attn_fwd_gqa with the addressing of
+ * flashd_splitk_partial_paged.  k_pages, v_pages : [num_pages, Hkv,
+ * page_size, d] bf16; page_size a multiple of 128 keys; block_table
+ * [B, max_pages] and seq_lens [B] int32 in DEVICE memory; q, o :
+ * [B, Hkv*G, Nq, d] bf16.  The Nq positions of sequence b are its last Nq
+ * (causal: position iq sees keys 0 .. seq_lens[b] - Nq + iq; a position
+ * that would see no key gives o = 0).  Split ranges are whole 128-key
+ * chunks of ceil(seq_lens[b] / num_splits) keys; workspace, combine, the
+ * handling of a bad table or length (device status word) and the other
+ * errors as for the calls they combine.  num_splits <= 0 in
+ * flashd_attn_fwd_gqa_paged selects flashd_gqa_num_splits(B, Hkv, G,
+ * max_pages*page_size, d).                                                */
+int flashd_gqa_partial_paged(const void* q, const void* k_pages, const void* v_pages,
+                             const int* block_table, const int* seq_lens,
+                             void* workspace, size_t workspace_bytes,
+                             int B, int Hkv, int G, int Nq, int max_pages, int page_size, int num_pages,
+                             int d, float scale, int causal, int num_splits, void* stream);
+int flashd_attn_fwd_gqa_paged(const void* q, const void* k_pages, const void* v_pages, void* o,
+                              const int* block_table, const int* seq_lens,
+                              void* workspace, size_t workspace_bytes,
+                              int B, int Hkv, int G, int Nq, int max_pages, int page_size, int num_pages,
+                              int d, float scale, int causal, int num_splits, void* stream);
+
+/* ------------------------------------------------------------------------
  * Split-K forward that allocates nothing.  (The paper has no counterpart: this
  * entry point exists for integration reasons only.)
  *

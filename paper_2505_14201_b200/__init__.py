@@ -12,6 +12,6 @@ from .binding import (  # noqa: F401
     flashd_splitk_combine, flashd_attn_fwd_splitk, flashd_attn_fwd_splitk_static, flashd_attn_fwd_host,
     flashd_gqa_num_splits, flashd_gqa_partial, flashd_attn_fwd_gqa, MAX_GROUP,
     flashd_attn_fwd_pwl, PWL_MAX_SEGMENTS, flashd_splitk_partial_fp8kv, flashd_attn_fwd_splitk_fp8kv,
-    flashd_splitk_partial_paged, flashd_attn_fwd_splitk_paged,
+    flashd_splitk_partial_paged, flashd_attn_fwd_splitk_paged, flashd_attn_fwd_gqa_paged,
     flashd_skip_stats, flashd_last_device_status, BF16, F32, MAX_SPLITS, STATIC_SCRATCH_BYTES, EXPORTED_SYMBOLS,
 )

@@ -22,6 +22,7 @@ EXPORTED_SYMBOLS = (
     "flashd_splitk_partial_fp8kv", "flashd_attn_fwd_splitk_fp8kv",
     "flashd_splitk_partial_paged", "flashd_attn_fwd_splitk_paged", "flashd_attn_fwd_fp8",
     "flashd_splitk_partial_paged_fp8kv", "flashd_attn_fwd_splitk_paged_fp8kv",
+    "flashd_gqa_partial_paged", "flashd_attn_fwd_gqa_paged",
     "flashd_attn_fwd_host", "flashd_skip_stats", "flashd_last_device_status", "flashd_status_string", "flashd_version", "flashd_launch_count",
 )
 
@@ -67,6 +68,8 @@ def lib() -> ctypes.CDLL:
             L.flashd_splitk_partial_paged.argtypes = [vp, vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_attn_fwd_splitk_paged.argtypes = [vp, vp, vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, ci, ci, cf, ci, vp]
             L.flashd_splitk_partial_paged_fp8kv.argtypes = L.flashd_splitk_partial_paged.argtypes
+            L.flashd_gqa_partial_paged.argtypes = [vp, vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, ci, ci, ci, cf, ci, ci, vp]
+            L.flashd_attn_fwd_gqa_paged.argtypes = [vp, vp, vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, ci, ci, ci, cf, ci, ci, vp]
             L.flashd_attn_fwd_splitk_paged_fp8kv.argtypes = L.flashd_attn_fwd_splitk_paged.argtypes
             fp = ctypes.POINTER(ctypes.c_float)
             L.flashd_attn_fwd_pwl.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, ci,
@@ -337,6 +340,33 @@ def flashd_attn_fwd_splitk_paged(q, k_pages, v_pages, block_table, seq_lens, sca
     _check(fn(_ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(o), _ptr(block_table), _ptr(seq_lens), _ptr(workspace),
               workspace.numel() * workspace.element_size(), B, H, Nq, max_pages, page_size, num_pages, d,
               float(scale), int(num_splits), _stream_ptr(stream)), "flashd_attn_fwd_splitk_paged")
+    return o
+
+
+def flashd_attn_fwd_gqa_paged(q, k_pages, v_pages, block_table, seq_lens, scale, num_splits=0, causal=False,
+                              workspace=None, o=None, stream=None):
+    """Grouped-query decode over a paged K/V pool (``q: [B,Hkv*G,Nq,d]``, pool ``[num_pages,Hkv,page_size,d]``)."""
+    import torch
+    for t in (q, k_pages, v_pages, block_table, seq_lens):
+        if not t.is_contiguous():
+            raise ValueError("paged grouped-query decode: all tensors must be contiguous")
+    B, Hq, Nq, d = q.shape
+    num_pages, Hkv, page_size, dk = k_pages.shape
+    if dk != d or Hq % Hkv != 0 or tuple(v_pages.shape) != tuple(k_pages.shape) or block_table.shape[0] != B \
+            or tuple(seq_lens.shape) != (B,) or block_table.dtype != torch.int32 or seq_lens.dtype != torch.int32:
+        raise ValueError("paged grouped-query decode: shapes or dtypes do not match")
+    G = Hq // Hkv
+    max_pages = block_table.shape[1]
+    S = num_splits if num_splits > 0 else flashd_gqa_num_splits(B, Hkv, G, max_pages * page_size, d)
+    if workspace is None:
+        workspace = torch.empty((B, Hq, Nq, max(S, 1), d + 1), dtype=torch.float32, device=q.device)
+    if o is None:
+        o = torch.empty_like(q)
+    _check(lib().flashd_attn_fwd_gqa_paged(_ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(o), _ptr(block_table),
+                                           _ptr(seq_lens), _ptr(workspace),
+                                           workspace.numel() * workspace.element_size(), B, Hkv, G, Nq, max_pages,
+                                           page_size, num_pages, d, float(scale), int(bool(causal)), int(num_splits),
+                                           _stream_ptr(stream)), "flashd_attn_fwd_gqa_paged")
     return o
 
 

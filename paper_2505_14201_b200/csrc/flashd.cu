@@ -221,17 +221,20 @@ int launch_partial(const void* q, const void* k, const void* v, void* ws, long l
     return after_launch();
 }
 
-template <int D>
+template <int D, bool PAGED = false>
 int launch_gqa_partial(const void* q, const void* k, const void* v, void* ws, int BHkv, int R, int Nq, int causal,
-                       int Nk, float scale, int num_splits, cudaStream_t stream) {
+                       int Nk, float scale, int num_splits, cudaStream_t stream, const PagedKV& pg = PagedKV{}) {
     using C = GqaCfg<D>;
     CUtensorMap mk, mv;
-    if (!make_map(&mk, k, BHkv, Nk, D) || !make_map(&mv, v, BHkv, Nk, D)) return FLASHD_ERR_CUDA;
+    // contiguous: (D, Nk, B*Hkv); paged: the pool as (D, page_size, num_pages*Hkv)
+    const int slabs = PAGED ? pg.num_pages * pg.H : BHkv;
+    const int rows_per_slab = PAGED ? pg.page_size : Nk;
+    if (!make_map(&mk, k, slabs, rows_per_slab, D) || !make_map(&mv, v, slabs, rows_per_slab, D)) return FLASHD_ERR_CUDA;
     static bool attr_set[64] = {false};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FLASHD_ERR_CUDA;
     if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(gqa_partial_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(gqa_partial_kernel<D, PAGED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  C::kSmemBytes) != cudaSuccess)
             return FLASHD_ERR_CUDA;
         attr_set[dev] = true;
@@ -240,9 +243,9 @@ int launch_gqa_partial(const void* q, const void* k, const void* v, void* ws, in
     if (sms <= 0) return FLASHD_ERR_CUDA;
     const long long items = (long long)BHkv * num_splits;
     const int grid = (int)(items < sms ? items : sms);
-    gqa_partial_kernel<D><<<grid, C::kThreads, C::kSmemBytes, stream>>>(
+    gqa_partial_kernel<D, PAGED><<<grid, C::kThreads, C::kSmemBytes, stream>>>(
         mk, mv, static_cast<const __nv_bfloat16*>(q), static_cast<float*>(ws), BHkv, R, Nq, causal, Nk,
-        scale * kLog2e, num_splits);
+        scale * kLog2e, num_splits, pg);
     return after_launch();
 }
 
@@ -599,6 +602,55 @@ int flashd_attn_fwd_gqa(const void* q, const void* k, const void* v, void* o, vo
     if (num_splits <= 0) num_splits = flashd_gqa_num_splits(B, Hkv, G, Nk, d);
     const int st = flashd_gqa_partial(q, k, v, workspace, workspace_bytes, B, Hkv, G, Nq, Nk, d, scale, causal,
                                       num_splits, stream);
+    if (st != FLASHD_OK) return st;
+    return flashd_splitk_combine(workspace, o, nullptr, B, Hkv * G, Nq, d, num_splits, FLASHD_BF16, stream);
+}
+
+int flashd_gqa_partial_paged(const void* q, const void* k_pages, const void* v_pages, const int* block_table,
+                             const int* seq_lens, void* workspace, size_t workspace_bytes, int B, int Hkv, int G,
+                             int Nq, int max_pages, int page_size, int num_pages, int d, float scale, int causal,
+                             int num_splits, void* stream) {
+    if (!q || !k_pages || !v_pages || !block_table || !seq_lens || !workspace) return FLASHD_ERR_NULL;
+    if (B <= 0 || Hkv <= 0 || G < 1 || Nq < 1 || max_pages <= 0 || page_size <= 0 || num_pages <= 0 || d <= 0 ||
+        !std::isfinite(scale))
+        return FLASHD_ERR_SHAPE;
+    if ((long long)G * Nq > FLASHD_MAX_GROUP) return FLASHD_ERR_UNSUPPORTED;
+    if ((long long)max_pages * page_size > 0x7fffffffLL || (long long)num_pages * Hkv > 0x7fffffffLL) return FLASHD_ERR_SHAPE;
+    if ((long long)B * Hkv * G > 0x7fffffffLL / FLASHD_MAX_SPLITS) return FLASHD_ERR_SHAPE;
+    if (!aligned16(q) || !aligned16(k_pages) || !aligned16(v_pages) || !aligned16(workspace) ||
+        (reinterpret_cast<uintptr_t>(block_table) & 3u) || (reinterpret_cast<uintptr_t>(seq_lens) & 3u))
+        return FLASHD_ERR_ALIGN;
+    if (d != 128 && d != 64) return FLASHD_ERR_UNSUPPORTED;
+    if (page_size % 128 != 0) return FLASHD_ERR_UNSUPPORTED;        // a 128-key chunk must not straddle pages
+    if (num_splits < 1 || num_splits > FLASHD_MAX_SPLITS) return FLASHD_ERR_WORKSPACE;
+    if (workspace_bytes < flashd_splitk_workspace_bytes(B, Hkv * G, Nq, d, num_splits)) return FLASHD_ERR_WORKSPACE;
+    PagedKV pg;
+    pg.block_table = block_table;
+    pg.seq_lens = seq_lens;
+    pg.max_pages = max_pages;
+    pg.page_size = page_size;
+    pg.num_pages = num_pages;
+    pg.H = Hkv;
+    const int cz = causal ? 1 : 0;
+    if (d == 128)
+        return launch_gqa_partial<128, true>(q, k_pages, v_pages, workspace, B * Hkv, G * Nq, Nq, cz, 0, scale, num_splits,
+                                             as_stream(stream), pg);
+    return launch_gqa_partial<64, true>(q, k_pages, v_pages, workspace, B * Hkv, G * Nq, Nq, cz, 0, scale, num_splits,
+                                        as_stream(stream), pg);
+}
+
+int flashd_attn_fwd_gqa_paged(const void* q, const void* k_pages, const void* v_pages, void* o,
+                              const int* block_table, const int* seq_lens, void* workspace, size_t workspace_bytes,
+                              int B, int Hkv, int G, int Nq, int max_pages, int page_size, int num_pages, int d,
+                              float scale, int causal, int num_splits, void* stream) {
+    if (!o) return FLASHD_ERR_NULL;
+    if (!aligned16(o)) return FLASHD_ERR_ALIGN;
+    if (num_splits <= 0 && B > 0 && Hkv > 0 && G > 0 && max_pages > 0 && page_size > 0 &&
+        (long long)max_pages * page_size <= 0x7fffffffLL)
+        num_splits = flashd_gqa_num_splits(B, Hkv, G, max_pages * page_size, d);
+    const int st = flashd_gqa_partial_paged(q, k_pages, v_pages, block_table, seq_lens, workspace, workspace_bytes, B,
+                                            Hkv, G, Nq, max_pages, page_size, num_pages, d, scale, causal, num_splits,
+                                            stream);
     if (st != FLASHD_OK) return st;
     return flashd_splitk_combine(workspace, o, nullptr, B, Hkv * G, Nq, d, num_splits, FLASHD_BF16, stream);
 }

@@ -72,11 +72,16 @@ __device__ __forceinline__ void mma_rows8(float& d0, float& d1, uint32_t a0, uin
         : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.f));
 }
 
-template <int D>
+// PAGED = true: K and V live in a page pool [num_pages, Hkv, page_size, D] (the tensor maps then
+// cover (D, page_size, num_pages * Hkv)), sequence b owns the pages block_table[b][..] and has
+// seq_lens[b] keys; split ranges are whole 128-key chunks, so a chunk never straddles two pages.
+// Rows of a page past the sequence's end hold whatever the pool held: their weights are exactly
+// zero, and their V entries are cleared in registers so that 0 x NaN cannot reach the output.
+template <int D, bool PAGED = false>
 __global__ void __launch_bounds__(GqaCfg<D>::kThreads, 1)
 gqa_partial_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                    const __nv_bfloat16* __restrict__ q, float* __restrict__ workspace, int BHkv, int R, int Nq,
-                   int causal, int Nk, float scale_log2e, int num_splits) {
+                   int causal, int Nk, float scale_log2e, int num_splits, const PagedKV pg) {
     using C = GqaCfg<D>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // swizzle atoms: 1 KB
@@ -107,18 +112,44 @@ gqa_partial_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
             const int bh = (int)(item / num_splits);
             const int split = (int)(item - (long long)bh * num_splits);
-            const int k0 = split * per_split;
-            const int k1 = min(k0 + per_split, Nk);
+            int seq_nk = Nk, head = 0;
+            const int* pages = nullptr;
+            if (PAGED) {
+                const int b = bh / pg.H;
+                head = bh - b * pg.H;
+                seq_nk = pg.seq_lens[b];
+                pages = pg.block_table + (long long)b * pg.max_pages;
+                if (seq_nk < 0 || seq_nk > pg.max_pages * pg.page_size) {
+                    if (atomicCAS(&g_status[0], 0u, (unsigned int)FLASHD_ERR_SHAPE) == 0u) {
+                        g_status[1] = blockIdx.x; g_status[2] = kBadPageTable; g_status[3] = (unsigned int)b;
+                    }
+                    seq_nk = 0;
+                }
+            }
+            int k0, k1;
+            split_range<C::kChunk, PAGED>(seq_nk, num_splits, per_split, split, k0, k1);
             for (int c0 = k0; c0 < k1; c0 += C::kChunk, ++it) {
                 const int stage = it % C::kStages;
                 const uint32_t round = it / C::kStages;
                 if (round > 0 && !mbar_wait(&empty[stage], (round - 1) & 1, kWaitGqaEmpty)) return;
                 unsigned char* dst = ring + stage * C::kStageBytes;
+                int row0 = c0, slab = bh;
+                if (PAGED) {
+                    int page = pages[c0 / pg.page_size];
+                    if ((unsigned int)page >= (unsigned int)pg.num_pages) {
+                        if (atomicCAS(&g_status[0], 0u, (unsigned int)FLASHD_ERR_SHAPE) == 0u) {
+                            g_status[1] = blockIdx.x; g_status[2] = kBadPageTable; g_status[3] = (unsigned int)page;
+                        }
+                        page = 0;
+                    }
+                    row0 = c0 % pg.page_size;
+                    slab = page * pg.H + head;
+                }
                 mbar_arrive_expect_tx(&full[stage], C::kStageBytes);
 #pragma unroll
                 for (int p = 0; p < C::kPanels; ++p) {
-                    tma_load_3d(dst + p * C::kPanelBytes, &map_k, p * 64, c0, bh, &full[stage]);
-                    tma_load_3d(dst + C::kTileBytes + p * C::kPanelBytes, &map_v, p * 64, c0, bh, &full[stage]);
+                    tma_load_3d(dst + p * C::kPanelBytes, &map_k, p * 64, row0, slab, &full[stage]);
+                    tma_load_3d(dst + C::kTileBytes + p * C::kPanelBytes, &map_v, p * 64, row0, slab, &full[stage]);
                 }
             }
         }
@@ -129,7 +160,7 @@ gqa_partial_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     const int grow = lane >> 2;            // query row (head g, position iq: grow = g*Nq + iq) of this lane's accumulators
     // keys [0, row_lim) are visible to the row: all of them, or, causal, up to the row's own
     // position Nk - Nq + iq (the queries are the last Nq positions of the sequence)
-    const int row_lim = causal ? Nk - Nq + (grow % Nq) + 1 : Nk;
+    int row_lim = causal ? Nk - Nq + (grow % Nq) + 1 : Nk;
     const int quad = lane & 3;
     constexpr int KS = D / 16;             // k-steps of the score product = pairs of output column tiles
     // shared-memory offsets of this lane's matrix rows (within a K or V tile)
@@ -144,8 +175,14 @@ gqa_partial_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     for (long long item = blockIdx.x; item < n_items; item += gridDim.x, ++item_idx) {
         const int bh = (int)(item / num_splits);
         const int split = (int)(item - (long long)bh * num_splits);
-        const int k0 = split * per_split;
-        const int k1 = min(k0 + per_split, Nk);
+        int seq_nk = Nk;
+        if (PAGED) {
+            seq_nk = pg.seq_lens[bh / pg.H];
+            if (seq_nk < 0 || seq_nk > pg.max_pages * pg.page_size) seq_nk = 0;
+            row_lim = causal ? seq_nk - Nq + (grow % Nq) + 1 : seq_nk;
+        }
+        int k0, k1;
+        split_range<C::kChunk, PAGED>(seq_nk, num_splits, per_split, split, k0, k1);
 
         // Q fragments of the group: row grow, columns 16 ks + 2 quad (+8)
         uint32_t qa0[KS], qa2[KS];
@@ -217,12 +254,21 @@ gqa_partial_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
                 const uint32_t pa2 = pack_bf16x2(p[1][0] * inv, p[1][1] * inv);   // keys 8 + 2 quad, +1
 #pragma unroll
                 for (int n = 0; n < 2 * KS; ++n) { oacc[n][0] *= alpha; oacc[n][1] *= alpha; }
+                // V entries of keys past the sequence's end (this lane holds key rows 2 quad, 2 quad + 1
+                // of the warp's lower and upper eight keys, packed as bf16 pairs)
+                uint32_t vmask_lo = 0xffffffffu, vmask_hi = 0xffffffffu;
+                if (PAGED) {
+                    const int kb = c0 + warp * 16 + 2 * quad;
+                    vmask_lo = (kb < seq_nk ? 0x0000ffffu : 0u) | (kb + 1 < seq_nk ? 0xffff0000u : 0u);
+                    vmask_hi = (kb + 8 < seq_nk ? 0x0000ffffu : 0u) | (kb + 9 < seq_nk ? 0xffff0000u : 0u);
+                }
                 // ---- o += P V : output column tiles 2j, 2j+1 per matrix load
 #pragma unroll
                 for (int j = 0; j < KS; ++j) {
                     const int chunk = 2 * j + v_csel;
                     uint32_t b[4];
                     ldsm_x4_trans(vs_base + (chunk >> 3) * C::kPanelBytes + v_row * 128 + (((chunk & 7) ^ (v_row & 7)) << 4), b);
+                    if (PAGED) { b[0] &= vmask_lo; b[1] &= vmask_hi; b[2] &= vmask_lo; b[3] &= vmask_hi; }
                     mma_rows8(oacc[2 * j][0], oacc[2 * j][1], pa0, pa2, b[0], b[1]);
                     mma_rows8(oacc[2 * j + 1][0], oacc[2 * j + 1][1], pa0, pa2, b[2], b[3]);
                 }

@@ -144,3 +144,47 @@ def test_paged_fp8_pool_matches_oracle(flashd_lib, d, page_size, lens, H, Nq, sp
     st, detail = flashd_lib.flashd_last_device_status()
     assert st == 0, detail
     check(got, q, ks, vs, lens, sc, ("fp8", d, page_size))
+
+
+@pytest.mark.parametrize("d,page_size,lens,Hkv,G,Nq,causal,splits", [
+    (128, 128, [1, 127, 128, 129, 3000], 2, 4, 1, False, 0),
+    (128, 256, [5000, 0, 600, 255], 2, 8, 1, False, 3),
+    (128, 128, [2, 131, 1000], 3, 2, 2, True, 0),          # two positions per head, causal among themselves
+    (64, 128, [1, 128, 129, 2000], 2, 4, 2, True, 2),
+    (64, 256, [4100, 77], 1, 7, 1, False, 0),
+])
+def test_paged_grouped_query_matches_oracle(flashd_lib, d, page_size, lens, Hkv, G, Nq, causal, splits):
+    """G query heads per K/V head over the paged pool; page tails past a sequence's end hold NaN,
+    which must not reach the output (their weights are zero and their V entries are cleared)."""
+    sc = f32_scale(d)
+    k_pages, v_pages, table, seq_lens, ks, vs = build_pool(lens, Hkv, d, page_size, seed=21 + d + page_size + G)
+    nan = torch.tensor(float("nan"), dtype=torch.bfloat16)
+    for b, n in enumerate(lens):
+        if n % page_size:
+            last = table[b, (n - 1) // page_size]
+            k_pages[last, :, n % page_size:] = nan
+            v_pages[last, :, n % page_size:] = nan
+    B = len(lens)
+    q, _, _ = synth.random_qkv(B, Hkv * G, Nq, 1, d, seed=97)
+    got = flashd_lib.flashd_attn_fwd_gqa_paged(q.cuda(), k_pages.cuda(), v_pages.cuda(), table.cuda(),
+                                               seq_lens.cuda(), sc, splits, causal=causal)
+    st, detail = flashd_lib.flashd_last_device_status()
+    assert st == 0, detail
+    g = got.cpu()
+    assert torch.all(torch.isfinite(g.float()))
+    errs = []
+    for b, n in enumerate(lens):
+        for iq in range(Nq):
+            vis = n - Nq + iq + 1 if causal else n      # keys visible to this position
+            if vis <= 0:
+                assert torch.all(g[b, :, iq] == 0), (b, iq)
+                continue
+            kk = ks[b][:, :vis].repeat_interleave(G, dim=0)[None]
+            vv = vs[b][:, :vis].repeat_interleave(G, dim=0)[None]
+            want = oracle.attn_naive(q[b:b + 1, :, iq:iq + 1], kk, vv, sc, False)
+            err = np.abs(g[b:b + 1, :, iq:iq + 1].double().numpy() - want)
+            # the bf16 output grid is coarser than the bound above 2 in magnitude: half an ulp is 2^-9 |o|
+            assert np.all(err <= BF16_MAX + 2.0 ** -9 * np.abs(want)), (b, iq, n, err.max())
+            errs.append(err.ravel())
+    # the mean bound is a statement about a workload, not about a two-key sequence: taken over the batch
+    assert np.concatenate(errs).mean() <= BF16_MEAN
