@@ -70,7 +70,8 @@ typedef enum { FLASHD_BF16 = 0, FLASHD_F32 = 1 } flashd_dtype;
  * run on the 5th generation tensor cores (tcgen05.mma, accumulators in tensor
  * memory).
  *
- * q, o: [B,H,Nq,d] bf16; k, v: [B,H,Nk,d] bf16.  d must be 64 or 128.
+ * q, o: [B,H,Nq,d] bf16; k, v: [B,H,Nk,d] bf16.  d must be 64, 128 or 256
+ * (the hidden sizes of Sec. V-A that a 128-row tensor-core tile can take).
  * o must not overlap q, k or v.  Returns after the launch.               */
 int flashd_attn_fwd(const void* q, const void* k, const void* v, void* o,
                     int B, int H, int Nq, int Nk, int d, float scale, int causal,

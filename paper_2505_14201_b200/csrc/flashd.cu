@@ -112,7 +112,7 @@ int launch_prefill(const void* q, const void* k, const void* v, void* o, float* 
     prm.scale_log2e = scale * kLog2e;
     prm.causal = causal ? 1 : 0;
     prm.out_f32 = out_f32;
-    prm.n_qpairs = (Nq + 255) / 256;
+    prm.n_qpairs = (Nq + C::kItemRows - 1) / C::kItemRows;
     prm.n_work = BH * prm.n_qpairs;
     const int sms = sm_count();
     if (sms <= 0) return FLASHD_ERR_CUDA;
@@ -336,6 +336,7 @@ int flashd_attn_fwd_ex(const void* q, const void* k, const void* v, void* o, flo
     const int BH = B * H;
     if (d == 128) return launch_prefill<128>(q, k, v, o, lse_out, out_dtype == FLASHD_F32, BH, Nq, Nk, scale, causal, as_stream(stream));
     if (d == 64) return launch_prefill<64>(q, k, v, o, lse_out, out_dtype == FLASHD_F32, BH, Nq, Nk, scale, causal, as_stream(stream));
+    if (d == 256) return launch_prefill<256>(q, k, v, o, lse_out, out_dtype == FLASHD_F32, BH, Nq, Nk, scale, causal, as_stream(stream));
     return FLASHD_ERR_UNSUPPORTED;
 }
 

@@ -27,6 +27,8 @@
 // is L alone (l_t is L_t - ref_t in the linear domain), one reciprocal per row and
 // tile plays the part of the sigmoid's division.
 //
+// D = 256 runs the D = 128 schedule with a single query tile per CTA (warps 4-7 idle): the
+// accumulator of one tile takes 256 tensor-memory columns and one Q tile 64 KB.
 // Warp roles (16 warps): 0-3 weights of query tile 0, 4-7 weights of query tile 1,
 // 8-11 correction + epilogue, 12 MMA issue (whole warp in uniform control flow, one elected
 // lane issues), 13 TMA loads (one lane), 14-15 idle.
@@ -51,6 +53,10 @@ namespace flashd {
 template <int D, int EB = 2>
 struct PrefillCfg {
     static_assert(EB == 2 || (EB == 1 && D == 128), "E4M3 operands: D = 128 only");
+    // D = 256: one query tile per CTA (its accumulator alone takes 256 of the 512 tensor-memory
+    // columns, and one Q tile 64 KB of shared memory); D = 64, 128: two.
+    static constexpr int kQTiles = (D == 256) ? 1 : 2;
+    static constexpr int kItemRows = 128 * kQTiles;              // query rows of a work item
     static constexpr int kBlockM = 128;
     static constexpr int kBlockN = 128;
     static constexpr int kPanels = D * EB / 128;                 // 128-byte swizzle panels (64 bf16 / 128 E4M3 columns)
@@ -61,10 +67,10 @@ struct PrefillCfg {
     static constexpr int kPCols = 128 * EB / 4;                  // tensor-memory columns of P (packed)
     static constexpr int kPanelBytes = 128 * 128;                // 128 rows x 128 bytes
     static constexpr int kTileBytes = kPanels * kPanelBytes;     // one Q / K / V tile
-    static constexpr int kStages = (D == 128) ? 4 : 6;           // K/V ring
+    static constexpr int kStages = (D == 256) ? 2 : (D == 128) ? 4 : 6;   // K/V ring (tiles of 16 KB x panels)
     static constexpr int kThreads = 512;
     static constexpr int kBarriers = 22 + 2 * kStages;
-    static constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + 3 * 2 * 128 * 4 + kBarriers * 8 + 64 + 1024;
+    static constexpr int kSmemBytes = kQTiles * kTileBytes + kStages * kTileBytes + 3 * 2 * 128 * 4 + kBarriers * 8 + 64 + 1024;
     static constexpr uint32_t kTmemCols = 512;
     // At D = 64 tensor memory has room for P next to S (S0 S1 P0 P1 O0 O1 = 512 columns), so
     // the score product of step t+1 can run while the weights of step t are computed
@@ -221,7 +227,7 @@ struct PrefillParams {
     float scale_log2e;  // scale * log2(e)
     int causal;
     int out_f32;
-    int n_qpairs;       // ceil(Nq / 256)
+    int n_qpairs;       // ceil(Nq / rows of a work item)
     int n_work;         // BH * n_qpairs
 };
 
@@ -270,7 +276,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // 1024-byte alignment for the swizzled tiles
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     unsigned char* sQ = smem;                               // 2 tiles
-    unsigned char* sKV = smem + 2 * C::kTileBytes;          // kStages tiles
+    unsigned char* sKV = smem + C::kQTiles * C::kTileBytes; // kStages tiles
     // Per-row factors handed from the weights warps to the correction warps, [slot][tile][row].
     // Two slots used alternately: message n of a tile is written only after the product that
     // needed message n-1 has been issued, and that product waits for the correction warps to
@@ -358,8 +364,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 if (work_index(nw + 1) >= prm.n_work) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
                 const int qpair = prm.n_qpairs - 1 - w / prm.BH;
                 const int bh = w % prm.BH;
-                const int q0 = qpair * 256;
-                const int T0 = n_tiles(q0), T1 = n_tiles(q0 + 128);
+                const int q0 = qpair * C::kItemRows;
+                const int T0 = n_tiles(q0), T1 = (C::kQTiles == 2) ? n_tiles(q0 + 128) : 0;
                 const int T = max(T0, T1);
                 for (int i = 0; i < 2; ++i) {
                     if ((i == 0 ? T0 : T1) == 0) continue;
@@ -443,8 +449,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             bool early0 = false;        // S_0(0) of the work item about to start has been issued already
             for (int nw = 0, w = work_index(0); w < prm.n_work; w = work_index(++nw)) {
                 const int qpair = prm.n_qpairs - 1 - w / prm.BH;
-                const int q0 = qpair * 256;
-                const int T0 = n_tiles(q0), T1 = n_tiles(q0 + 128);
+                const int q0 = qpair * C::kItemRows;
+                const int T0 = n_tiles(q0), T1 = (C::kQTiles == 2) ? n_tiles(q0 + 128) : 0;
                 const int T = max(T0, T1);
                 auto stage_of = [&](uint32_t it) { return (int)(it % C::kStages); };
                 auto parity_of = [&](uint32_t it) { return (it / C::kStages) & 1u; };
@@ -535,7 +541,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         // it pulls the two tiles into phase, which costs more than it saves (c3: -2.5 %).
                         const int wn = work_index(nw + 1);
                         if (wn < prm.n_work) {
-                            const int T0n = n_tiles((prm.n_qpairs - 1 - wn / prm.BH) * 256);
+                            const int T0n = n_tiles((prm.n_qpairs - 1 - wn / prm.BH) * C::kItemRows);
                             const uint32_t it_k0 = kv_it + 2 * T;
                             if (T0n > 0 && mbar_test(&q_full[0], n_qf0 & 1) &&
                                 mbar_test(&kv_full[stage_of(it_k0)], parity_of(it_k0))) {
@@ -609,8 +615,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         for (int nw = 0, w = work_index(0); w < prm.n_work; w = work_index(++nw)) {
             const int qpair = prm.n_qpairs - 1 - w / prm.BH;
             const int bh = w % prm.BH;
-            const int q0 = qpair * 256 + i * 128;
-            const int Ti = n_tiles(q0);
+            const int q0 = qpair * C::kItemRows + i * 128;
+            const int Ti = (i < C::kQTiles) ? n_tiles(q0) : 0;
             const int gi = q0 + row;                   // global query index of this thread's row
             const int limit = prm.causal ? min(Nk, gi + 1) : Nk;   // keys [0, limit) are visible
             float L = -INFINITY;                       // log2-domain state: L = (s_i - ln w_i) * log2(e)
@@ -754,8 +760,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         for (int nw = 0, w = work_index(0); w < prm.n_work; w = work_index(++nw)) {
             const int qpair = prm.n_qpairs - 1 - w / prm.BH;
             const int bh = w % prm.BH;
-            const int q0 = qpair * 256;
-            const int Ti[2] = {n_tiles(q0), n_tiles(q0 + 128)};
+            const int q0 = qpair * C::kItemRows;
+            const int Ti[2] = {n_tiles(q0), (C::kQTiles == 2) ? n_tiles(q0 + 128) : 0};
             const int T = max(Ti[0], Ti[1]);
             // the O accumulators are free (the previous epilogue has read them)
             for (int i = 0; i < 2; ++i)

@@ -23,7 +23,7 @@ def test_random_shapes(flashd_lib):
     rnd = random.Random(1234)
     F8 = torch.float8_e4m3fn
     for it in range(150):
-        d = rnd.choice([64, 128])
+        d = rnd.choice([64, 128, 256])
         B = rnd.randint(1, 3)
         H = rnd.randint(1, 40 if it % 7 == 0 else 6)
         Nq = rnd.choice(NQ)

@@ -173,6 +173,24 @@ def test_prefill_many_short_work_items(flashd_lib, shape):
     ok_status(flashd_lib)
 
 
+@pytest.mark.parametrize("shape", [(1, 1, 128, 128, False), (1, 2, 256, 256, True), (2, 3, 200, 333, False),
+                                   (1, 2, 1, 1, False), (1, 4, 777, 777, True), (1, 3, 1000, 300, True),
+                                   (1, 200, 130, 260, True), (2, 8, 1024, 1024, False)])
+def test_prefill_hidden_size_256(flashd_lib, shape):
+    """d = 256, the largest hidden size of Sec. V-A, on the tensor path (one query tile per CTA)."""
+    B, H, Nq, Nk, causal = shape
+    d = 256
+    q, k, v = synth.random_qkv(B, H, Nq, Nk, d, seed=300 + Nq + Nk)
+    sc = f32_scale(d)
+    want, want_lse = oracle.attn_naive(q, k, v, sc, causal, return_lse=True)
+    qc, kc, vc = q.cuda(), k.cuda(), v.cuda()
+    got = flashd_lib.flashd_attn_fwd(qc, kc, vc, sc, causal)
+    got32, lse = flashd_lib.flashd_attn_fwd_ex(qc, kc, vc, sc, causal, out_dtype=torch.float32, return_lse=True)
+    ok_status(flashd_lib)
+    check_tiled(got, got32, want, shape)
+    assert np.abs(lse.double().cpu().numpy() - want_lse).max() <= 2e-3
+
+
 @pytest.mark.parametrize("d", [16, 256])
 @pytest.mark.parametrize("causal", [False, True])
 def test_perkey_hidden_sizes_of_the_paper(flashd_lib, d, causal):
