@@ -141,7 +141,7 @@ int flashd_attn_fwd_pwl(const void* q, const void* k, const void* v, void* o,
  * Tiled tensor-core forward with FP8-E4M3 operands (the second number format
  * of the paper's evaluation, Sec. V-A): q, k, v hold one-byte E4M3 values
  * (4 exponent bits, bias 7, 3 mantissa bits, no infinities), [B,H,N,d]
- * contiguous, 16-byte aligned; d = 128 only.  Same kernel and same steps as
+ * contiguous, 16-byte aligned; d = 128 or 256.  Same kernel and same steps as
  * flashd_attn_fwd (tile form of Algorithm 3, state L per row in fp32): both
  * products run as E4M3 x E4M3 -> fp32 on the tensor cores, the scores, the
  * weights' exponentials and row sums and the accumulator stay fp32, and the
@@ -155,7 +155,7 @@ int flashd_attn_fwd_pwl(const void* q, const void* k, const void* v, void* o,
  * o: bf16 or fp32 (out_dtype); lse_out nullable, [B,H,Nq] fp32, = L_N.
  * Dequantisation scales: one of Q and K folds into `scale`; one of V
  * multiplies the output and is the caller's.  Errors as flashd_attn_fwd_ex;
- * d != 128 returns FLASHD_ERR_UNSUPPORTED.                                 */
+ * any other d returns FLASHD_ERR_UNSUPPORTED.                             */
 int flashd_attn_fwd_fp8(const void* q, const void* k, const void* v, void* o,
                         float* lse_out, int out_dtype,
                         int B, int H, int Nq, int Nk, int d, float scale, int causal,

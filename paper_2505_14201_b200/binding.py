@@ -169,7 +169,7 @@ def flashd_attn_fwd_ex(q, k, v, scale, causal=False, out_dtype=None, return_lse=
 
 
 def flashd_attn_fwd_fp8(q, k, v, scale, causal=False, out_dtype=None, return_lse=False, o=None, stream=None):
-    """Tiled tensor-core forward with E4M3 operands (``torch.float8_e4m3fn`` q, k, v; d = 128);
+    """Tiled tensor-core forward with E4M3 operands (``torch.float8_e4m3fn`` q, k, v; d = 128 or 256);
     output bf16 (default) or fp32."""
     import torch
     B, H, Nq, Nk, d = _dims(q, k, v)

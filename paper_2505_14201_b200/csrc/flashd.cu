@@ -345,8 +345,11 @@ int flashd_attn_fwd_fp8(const void* q, const void* k, const void* v, void* o, fl
     const int st = check_common(q, k, v, o, B, H, Nq, Nk, d, scale);
     if (st != FLASHD_OK) return st;
     if (out_dtype != FLASHD_BF16 && out_dtype != FLASHD_F32) return FLASHD_ERR_UNSUPPORTED;
-    if (d != 128 || scale == 0.f) return FLASHD_ERR_UNSUPPORTED;
+    if ((d != 128 && d != 256) || scale == 0.f) return FLASHD_ERR_UNSUPPORTED;
     if (o == q || o == k || o == v) return FLASHD_ERR_SHAPE;
+    if (d == 256)
+        return launch_prefill<256, 1>(q, k, v, o, lse_out, out_dtype == FLASHD_F32, B * H, Nq, Nk, scale, causal,
+                                      as_stream(stream));
     return launch_prefill<128, 1>(q, k, v, o, lse_out, out_dtype == FLASHD_F32, B * H, Nq, Nk, scale, causal,
                                   as_stream(stream));
 }

@@ -35,7 +35,7 @@
 // Tensor memory (512 columns), D = 128: S0 | S1 | O0 | O1, P_i overlays the first 64
 // columns of S_i as packed bf16 pairs and is handed to the P V product in two halves of 64
 // keys; D = 64: S0 | S1 | P0 | P1 | O0 | O1.
-// Operands: bf16 (tcgen05.mma kind::f16) or FP8-E4M3 (kind::f8f6f4, D = 128; the weights are then
+// Operands: bf16 (tcgen05.mma kind::f16) or FP8-E4M3 (kind::f8f6f4, D = 128 or 256; the weights are then
 // stored as E4M3 with a per-row power-of-two scale, see the weights warps).
 // Every mbarrier wait is bounded; a wait that runs out records itself in the
 // device status word, raises the CTA's abort flag and the CTA drains and exits.
@@ -48,11 +48,11 @@
 namespace flashd {
 
 // EB = bytes per element of Q, K, V and P: 2 (bf16, tcgen05.mma kind::f16) or 1 (FP8-E4M3,
-// kind::f8f6f4; D = 128 only).  A product instruction covers 32 bytes of the contraction
+// kind::f8f6f4; D = 128 or 256).  A product instruction covers 32 bytes of the contraction
 // dimension: 16 bf16 or 32 E4M3 elements.
 template <int D, int EB = 2>
 struct PrefillCfg {
-    static_assert(EB == 2 || (EB == 1 && D == 128), "E4M3 operands: D = 128 only");
+    static_assert(EB == 2 || (EB == 1 && (D == 128 || D == 256)), "E4M3 operands: D = 128 or 256");
     // D = 256: one query tile per CTA (its accumulator alone takes 256 of the 512 tensor-memory
     // columns, and one Q tile 64 KB of shared memory); D = 64, 128: two.
     static constexpr int kQTiles = (D == 256) ? 1 : 2;
@@ -67,7 +67,7 @@ struct PrefillCfg {
     static constexpr int kPCols = 128 * EB / 4;                  // tensor-memory columns of P (packed)
     static constexpr int kPanelBytes = 128 * 128;                // 128 rows x 128 bytes
     static constexpr int kTileBytes = kPanels * kPanelBytes;     // one Q / K / V tile
-    static constexpr int kStages = (D == 256) ? 2 : (D == 128) ? 4 : 6;   // K/V ring (tiles of 16 KB x panels)
+    static constexpr int kStages = (D * EB == 512) ? 2 : (D == 64) ? 6 : 4;   // K/V ring (tiles of 16 KB x panels)
     static constexpr int kThreads = 512;
     static constexpr int kBarriers = 22 + 2 * kStages;
     static constexpr int kSmemBytes = kQTiles * kTileBytes + kStages * kTileBytes + 3 * 2 * 128 * 4 + kBarriers * 8 + 64 + 1024;

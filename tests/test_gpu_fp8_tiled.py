@@ -56,6 +56,18 @@ def test_fp8_tiled_shapes(flashd_lib, shape):
     assert torch.equal(got16, got32.to(torch.bfloat16))      # the bf16 output is the rounding of the fp32 one
 
 
+@pytest.mark.parametrize("shape", [(1, 1, 128, 128, False), (1, 2, 256, 256, True), (2, 3, 200, 333, False),
+                                   (1, 2, 1, 1, False), (1, 4, 777, 777, True), (1, 200, 130, 260, True)])
+def test_fp8_tiled_hidden_size_256(flashd_lib, shape):
+    B, H, Nq, Nk, causal = shape
+    d = 256
+    q, k, v = fp8_qkv(B, H, Nq, Nk, d, seed=700 + Nq + Nk)
+    sc = f32_scale(d)
+    got32 = flashd_lib.flashd_attn_fwd_fp8(q.cuda(), k.cuda(), v.cuda(), sc, causal, out_dtype=torch.float32)
+    ok_status(flashd_lib)
+    check(got32, q, k, v, sc, causal, shape)
+
+
 def test_equal_scores_give_the_mean_of_every_code(flashd_lib):
     """K = 0: every weight is exactly 1 (representable), so the output is the plain mean of the V
     rows and only fp32 accumulation rounds.  V runs through all 254 finite E4M3 codes."""

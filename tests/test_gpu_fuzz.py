@@ -43,7 +43,7 @@ def test_random_shapes(flashd_lib):
         assert torch.isfinite(a).all(), what
         assert torch.equal(a, a2), what
         assert (a - ref).abs().max().item() <= 1e-2, what
-        if d == 128 and it % 3 == 0:
+        if d >= 128 and it % 3 == 0:
             q8, k8, v8 = q.to(F8), k.to(F8), v.to(F8)
             o8 = flashd_lib.flashd_attn_fwd_fp8(q8, k8, v8, sc, causal, out_dtype=torch.float32)
             o8b = flashd_lib.flashd_attn_fwd_fp8(q8, k8, v8, sc, causal, out_dtype=torch.float32)
