@@ -27,8 +27,9 @@
 // is L alone (l_t is L_t - ref_t in the linear domain), one reciprocal per row and
 // tile plays the part of the sigmoid's division.
 //
-// D = 256 runs the D = 128 schedule with a single query tile per CTA (warps 4-7 idle): the
-// accumulator of one tile takes 256 tensor-memory columns and one Q tile 64 KB.
+// D = 256 runs a single query tile per CTA (warps 4-7 idle): the accumulator of one tile takes
+// 256 tensor-memory columns and one Q tile 64 KB.  The scores then alternate between the two S
+// regions, so that S(t+1) is computed under the weights of step t and P V(t) under those of t+1.
 // Warp roles (16 warps): 0-3 weights of query tile 0, 4-7 weights of query tile 1,
 // 8-11 correction + epilogue, 12 MMA issue (whole warp in uniform control flow, one elected
 // lane issues), 13 TMA loads (one lane), 14-15 idle.
@@ -57,6 +58,12 @@ struct PrefillCfg {
     // columns, and one Q tile 64 KB of shared memory); D = 64, 128: two.
     static constexpr int kQTiles = (D == 256) ? 1 : 2;
     static constexpr int kItemRows = 128 * kQTiles;              // query rows of a work item
+    // With one query tile the second S region is free: the scores alternate between the two
+    // S regions step by step (P overlaying the region its scores came from), S(t+1) is computed
+    // under the weights of step t and P V(t) under those of step t+1.  Everything indexed by
+    // query tile in the two-tile schedule (S/P regions, s_full, p_half, p_full, alpha_full and
+    // the slots of the per-row factors) is then indexed by the parity of the step.
+    static constexpr bool kAltS = (kQTiles == 1);
     static constexpr int kBlockM = 128;
     static constexpr int kBlockN = 128;
     static constexpr int kPanels = D * EB / 128;                 // 128-byte swizzle panels (64 bf16 / 128 E4M3 columns)
@@ -376,16 +383,25 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         tma_load_3d(sQ + i * C::kTileBytes + p * C::kPanelBytes, &map_q, p * C::kPanelCols, q0 + i * 128, bh,
                                     &q_full[i]);
                 }
-                for (int t = 0; t < T; ++t) {
-                    for (int kv = 0; kv < 2; ++kv, ++kv_it) {
-                        const int stage = kv_it % C::kStages;
-                        const uint32_t round = kv_it / C::kStages;
-                        if (round > 0 && !pf_wait(&kv_empty[stage], (round - 1) & 1, kWaitKVEmpty, abort_flag)) goto done;
-                        mbar_arrive_expect_tx(&kv_full[stage], C::kTileBytes);
-                        for (int p = 0; p < C::kPanels; ++p)
-                            tma_load_3d(sKV + stage * C::kTileBytes + p * C::kPanelBytes, kv == 0 ? &map_k : &map_v,
-                                        p * C::kPanelCols, t * 128, bh, &kv_full[stage]);
+                // ring order = order of use: K0 V0 K1 V1 ... (two tiles), K0 K1 V0 K2 V1 ... (alternating S)
+                for (int n = 0; n < 2 * T; ++n, ++kv_it) {
+                    int kv = n & 1, t = n >> 1;
+                    if (C::kAltS) {
+                        if (n < 2 && n < T) { kv = 0; t = n; }                       // K0, K1
+                        else {
+                            const int m = n - min(T, 2);                             // V0 K2 V1 K3 ... then the last V's
+                            const int pairs = max(T - 2, 0);                         // (V, K) pairs
+                            if (m < 2 * pairs) { kv = (m & 1) ? 0 : 1; t = (m & 1) ? (m >> 1) + 2 : (m >> 1); }
+                            else { kv = 1; t = pairs + (m - 2 * pairs); }
+                        }
                     }
+                    const int stage = kv_it % C::kStages;
+                    const uint32_t round = kv_it / C::kStages;
+                    if (round > 0 && !pf_wait(&kv_empty[stage], (round - 1) & 1, kWaitKVEmpty, abort_flag)) goto done;
+                    mbar_arrive_expect_tx(&kv_full[stage], C::kTileBytes);
+                    for (int p = 0; p < C::kPanels; ++p)
+                        tma_load_3d(sKV + stage * C::kTileBytes + p * C::kPanelBytes, kv == 0 ? &map_k : &map_v,
+                                    p * C::kPanelCols, t * 128, bh, &kv_full[stage]);
                 }
             }
         }
@@ -419,7 +435,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 const uint32_t ka = k_lo0 + stage * (C::kTileBytes >> 4);
 #pragma unroll
                 for (int ks = 0; ks < KS; ++ks) {
-                    if (leader) mma_ss64<EB>(tS[i], desc64(q_lo[i] + koff(ks), desc_hi), desc64(ka + koff(ks), desc_hi), idesc_s, ks > 0);
+                    if (leader) mma_ss64<EB>(tS[i], desc64(q_lo[C::kAltS ? 0 : i] + koff(ks), desc_hi), desc64(ka + koff(ks), desc_hi), idesc_s, ks > 0);
                     __syncwarp();
                     mid(ks * (8 / KS));
                 }
@@ -429,7 +445,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll
                 for (int kk = 0; kk < KP / 2; ++kk) {
                     const int ks = part * (KP / 2) + kk;
-                    if (leader) mma_ts64<EB>(tO[i], tP[i] + ks * 8, desc64(va + ks * (C::kVStepBytes >> 4), desc_hi), idesc_o, (!first) || ks > 0);
+                    if (leader) mma_ts64<EB>(tO[C::kAltS ? 0 : i], tP[i] + ks * 8, desc64(va + ks * (C::kVStepBytes >> 4), desc_hi), idesc_o, (!first) || ks > 0);
                     __syncwarp();
                 }
             };
@@ -447,6 +463,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 __syncwarp();
             };
             bool early0 = false;        // S_0(0) of the work item about to start has been issued already
+            uint32_t gstep = 0;         // steps so far on this CTA (alternating S: region of a step = its parity)
+            uint32_t n_sb[2] = {0, 0};  // alternating S: uses of p_half / p_full of each region
             for (int nw = 0, w = work_index(0); w < prm.n_work; w = work_index(++nw)) {
                 const int qpair = prm.n_qpairs - 1 - w / prm.BH;
                 const int q0 = qpair * C::kItemRows;
@@ -454,6 +472,51 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 const int T = max(T0, T1);
                 auto stage_of = [&](uint32_t it) { return (int)(it % C::kStages); };
                 auto parity_of = [&](uint32_t it) { return (it / C::kStages) & 1u; };
+                if constexpr (C::kAltS) {
+                    // ---- one query tile, scores alternating between the two S regions.
+                    // Order on the tensor pipe: S(0) S(1) | P V(0) S(2) | P V(1) S(3) | ...; S(t+2) goes
+                    // into the region P V(t) has just read P from (same issuing thread: in order).
+                    auto none1 = [](int) {};
+                    uint32_t r = kv_it;                      // ring position, in order of use
+                    for (int u = 0; u < 2 && u < T; ++u, ++r) {
+                        const int b = (int)((gstep + u) & 1);
+                        if (!pf_wait(&kv_full[stage_of(r)], parity_of(r), kWaitKVFull, abort_flag)) goto done;
+                        if (u == 0) { if (!pf_wait(&q_full[0], n_qf0 & 1, kWaitQFull, abort_flag)) goto done; ++n_qf0; }
+                        tc_fence_after();
+                        fire_S(b, stage_of(r), none1);
+                        commit(&s_full[b]);
+                        if (u + 1 == T) commit(&q_empty[0]);
+                        commit(&kv_empty[stage_of(r)]);
+                    }
+                    for (int t = 0; t < T; ++t) {
+                        const int b = (int)((gstep + t) & 1);
+                        if (!pf_wait(&kv_full[stage_of(r)], parity_of(r), kWaitKVFull, abort_flag)) goto done;
+                        if (!pf_wait(&o_ready[0], n_or0 & 1, kWaitOReady, abort_flag)) goto done;
+                        ++n_or0;
+                        if (!pf_wait(&p_half[b], n_sb[b] & 1, kWaitPFull, abort_flag)) goto done;
+                        tc_fence_after();
+                        fire_PV_part(b, stage_of(r), t == 0, 0);
+                        if (!pf_wait(&p_full[b], n_sb[b] & 1, kWaitPFull, abort_flag)) goto done;
+                        ++n_sb[b];
+                        tc_fence_after();
+                        fire_PV_part(b, stage_of(r), false, 1);
+                        commit(&pv_done[0]);
+                        commit(&kv_empty[stage_of(r)]);
+                        ++r;
+                        if (t + 2 < T) {
+                            if (!pf_wait(&kv_full[stage_of(r)], parity_of(r), kWaitKVFull, abort_flag)) goto done;
+                            tc_fence_after();
+                            fire_S(b, stage_of(r), none1);
+                            commit(&s_full[b]);
+                            if (t + 3 == T) commit(&q_empty[0]);
+                            commit(&kv_empty[stage_of(r)]);
+                            ++r;
+                        }
+                    }
+                    kv_it += 2 * T;
+                    gstep += T;
+                    continue;
+                }
                 // "known complete" flags of the next unconsumed phase of each barrier
                 uint32_t e_sf0 = 0, e_sf1 = 0, e_pf0 = 0, e_pf1 = 0, e_or0 = 0, e_or1 = 0, e_kvv = 0, e_kvk = 0;
                 auto none = [](int) {};
@@ -608,10 +671,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const int i = warp >> 2;                       // query tile of this warpgroup
         const int row = threadIdx.x & 127;             // row within the tile = tensor-memory lane
         const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tS = tmem_base + (i == 0 ? C::kColS0 : C::kColS1) + lane_sel;
-        const uint32_t tP = tmem_base + (i == 0 ? C::kColP0 : C::kColP1) + lane_sel;
         const float c = prm.scale_log2e;
-        uint32_t n_s = 0, n_ae = 0, n_pk = 0;
+        uint32_t n_s[2] = {0, 0}, n_ae = 0, n_pk = 0;
+        uint32_t gstep = 0;                            // steps so far (alternating S: region of a step = its parity)
         for (int nw = 0, w = work_index(0); w < prm.n_work; w = work_index(++nw)) {
             const int qpair = prm.n_qpairs - 1 - w / prm.BH;
             const int bh = w % prm.BH;
@@ -623,8 +685,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             float inv_l = 1.f;                         // 1 / l of the previous tile
             float K_prev = 0.f;                        // exponent offset of the stored weights (E4M3 only)
             for (int t = 0; t < Ti; ++t) {
-                if (!pf_wait(&s_full[i], n_s & 1, kWaitSFull, abort_flag)) goto done;
-                ++n_s;
+                // region of this step's scores and weights, and index of its barriers: the query
+                // tile, or, with one tile and alternating S regions, the parity of the step
+                const int bi = C::kAltS ? (int)((gstep + t) & 1) : i;
+                const uint32_t tS = tmem_base + (bi == 0 ? C::kColS0 : C::kColS1) + lane_sel;
+                const uint32_t tP = tmem_base + (bi == 0 ? C::kColP0 : C::kColP1) + lane_sel;
+                if (!pf_wait(&s_full[bi], n_s[bi] & 1, kWaitSFull, abort_flag)) goto done;
+                ++n_s[bi];
                 tc_fence_after();
                 float s[128];
 #pragma unroll
@@ -683,9 +750,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     K_prev = Kf;
                 }
                 if (C::kLookahead == 1 && t > 0) {
-                    sAlpha[(n_ae & 1) * 256 + i * 128 + row] = beta;
-                    ++n_ae;
-                    mbar_arrive(&alpha_full[i]);
+                    if (C::kAltS) {
+                        sAlpha[bi * 256 + row] = beta;       // slot and barrier of this step's parity
+                        mbar_arrive(&alpha_full[bi]);
+                    } else {
+                        sAlpha[(n_ae & 1) * 256 + i * 128 + row] = beta;
+                        ++n_ae;
+                        mbar_arrive(&alpha_full[i]);
+                    }
                 }
                 const uint64_t c2 = pack2(c, c), nref2 = pack2(Kf - ref, Kf - ref);
                 uint64_t acc0 = pack2(0.f, 0.f), acc1 = acc0;
@@ -698,7 +770,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                             // the first 64 weights are in tensor memory: their product may start
                             tc_wait_st();
                             tc_fence_before();
-                            mbar_arrive(&p_half[i]);
+                            mbar_arrive(&p_half[bi]);
                         }
                         float x0, x1, x2, x3;
                         unpack2(fma2(pack2(s[64 * h + j], s[64 * h + j + 1]), c2, nref2), x0, x1);
@@ -737,8 +809,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 L = ref + lg2(l);
                 tc_wait_st();
                 tc_fence_before();
-                mbar_arrive(&p_full[i]);
+                mbar_arrive(&p_full[bi]);
             }
+            gstep += Ti;
             if (Ti > 0) {
                 // the reciprocal that closes the last step goes to the epilogue.  The previous
                 // work item's message must have been consumed: for items of two or more tiles
@@ -757,6 +830,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tO[2] = {tmem_base + C::kColO0 + lane_sel, tmem_base + C::kColO1 + lane_sel};
         uint32_t n_af[2] = {0, 0}, n_pv[2] = {0, 0}, n_fin[2] = {0, 0};
+        uint32_t gstep_run = 0;                        // steps so far (alternating S: parity selects the factor's slot)
         for (int nw = 0, w = work_index(0); w < prm.n_work; w = work_index(++nw)) {
             const int qpair = prm.n_qpairs - 1 - w / prm.BH;
             const int bh = w % prm.BH;
@@ -766,12 +840,17 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             // the O accumulators are free (the previous epilogue has read them)
             for (int i = 0; i < 2; ++i)
                 if (Ti[i] > 0) { tc_fence_before(); mbar_arrive(&o_ready[i]); }
+            const uint32_t gstep = gstep_run;
+            gstep_run += (uint32_t)T;
             for (int t = 1; t < T; ++t) {
                 for (int i = 0; i < 2; ++i) {
                     if (t >= Ti[i]) continue;
-                    if (!pf_wait(&alpha_full[i], n_af[i] & 1, kWaitAlphaFull, abort_flag)) goto done;
-                    const float beta = sAlpha[(n_af[i] & 1) * 256 + i * 128 + row];
-                    ++n_af[i];
+                    // per-row factor of this step: slot and barrier of the query tile or, with
+                    // alternating S regions, of the step's parity
+                    const int ai = C::kAltS ? (int)((gstep + t) & 1) : i;
+                    if (!pf_wait(&alpha_full[ai], n_af[ai] & 1, kWaitAlphaFull, abort_flag)) goto done;
+                    const float beta = C::kAltS ? sAlpha[ai * 256 + row] : sAlpha[(n_af[i] & 1) * 256 + i * 128 + row];
+                    ++n_af[ai];
                     if (!pf_wait(&pv_done[i], n_pv[i] & 1, kWaitPVDone, abort_flag)) goto done;
                     ++n_pv[i];
                     tc_fence_after();
